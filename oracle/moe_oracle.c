@@ -1,0 +1,553 @@
+/*
+ * moe_oracle.c -- TEST INFRASTRUCTURE, not product code.
+ *
+ * A plain, slow, single-threaded CPU statement of what one forward pass of the
+ * fused block-scaled FP8 mixture-of-experts layer computes (the "Fused MoE"
+ * workload, Section "Kernel Design and Optimization / Fused MoE" of the paper:
+ * routing -> gather per expert -> FP8 GEMM1 -> SwiGLU -> re-quantisation ->
+ * FP8 GEMM2 -> weighted scatter back to token positions).
+ *
+ * Only tests, the smoke check and the benchmark's CPU-baseline leg may call
+ * this file.  It shares no code, header, table or constant generator with the
+ * CUDA path; the CUDA path never calls it.
+ *
+ * Arithmetic: fp32, round-to-nearest-even, no fused contraction except where
+ * fmaf() is written (build with -ffp-contract=off).  An optional fp64
+ * accumulation mode exists to measure this file's own rounding noise.
+ *
+ * Pins (tests that do not pass through this file's own formulas):
+ *   - FP8/bf16 codecs: every code against the library conversion of PyTorch.
+ *   - expdet/sigmoid: within 2 ulp of the fp64 library exp.
+ *   - routing: closed forms (uniform logits; planted winners), a hand-worked
+ *     miniature, a brute-force full sort, the weight-sum invariant.
+ *   - permutation: bijection + a library stable sort.
+ *   - MLP/combine: fp64 library matmul on dequantised tensors for the
+ *     single-expert closed form; identity-weight closed forms; exact scaling
+ *     and token-permutation invariants; the dense all-experts brute force in
+ *     this file (moe_ref_dense_bruteforce) is written separately from
+ *     moe_ref_forward and the two are compared.
+ *   - Parity with the PyTorch reference used by the paper's contest harness is
+ *     UNPINNED: that reference is not available and the paper prints no
+ *     numeric example for this workload.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define MOE_REF_OK 0
+#define MOE_REF_BAD_ARG (-1)
+#define MOE_REF_NO_MEM (-2)
+
+#define QBLOCK 128 /* quantisation block: 128 activations share one scale;    */
+                   /* weights carry one scale per 128x128 block (Fused MoE     */
+                   /* paragraph: "128-element blockwise FP32 scaling factors") */
+
+/* ------------------------------------------------------------------------ */
+/* Number formats                                                            */
+/* ------------------------------------------------------------------------ */
+
+/* FP8 e4m3 ("fn" flavour: no infinities, 0x7F/0xFF are NaN, largest finite
+ * value 448): 1 sign, 4 exponent bits with bias 7, 3 mantissa bits. */
+float moe_ref_e4m3_decode(uint8_t code)
+{
+    int s = code >> 7;
+    int e = (code >> 3) & 0xF;
+    int m = code & 0x7;
+    float v;
+    if (e == 0xF && m == 0x7)
+        return NAN;
+    if (e == 0)
+        v = ldexpf((float)m / 8.0f, -6);
+    else
+        v = ldexpf(1.0f + (float)m / 8.0f, e - 7);
+    return s ? -v : v;
+}
+
+/* fp32 -> e4m3, round to nearest, ties to even, magnitudes above 448 clamp to
+ * 448 (saturating), NaN -> 0x7F. */
+uint8_t moe_ref_e4m3_encode(float x)
+{
+    uint8_t sign = signbit(x) ? 0x80 : 0x00;
+    float a = fabsf(x);
+    int ex, m, E;
+    float f;
+    if (isnan(x))
+        return 0x7F;
+    if (a > 448.0f)
+        return sign | 0x7E;
+    if (a < 0.015625f) { /* below 2^-6: subnormal grid, spacing 2^-9 */
+        m = (int)nearbyintf(a * 512.0f); /* 0..8; 8 is the first normal code */
+        return sign | (uint8_t)m;
+    }
+    f = frexpf(a, &ex); /* a = f * 2^ex, f in [0.5, 1) */
+    E = ex - 1;         /* a = (2f) * 2^E, 2f in [1, 2) */
+    m = (int)nearbyintf((2.0f * f - 1.0f) * 8.0f);
+    if (m == 8) {
+        m = 0;
+        E += 1;
+    }
+    return sign | (uint8_t)(((E + 7) << 3) | m);
+}
+
+float moe_ref_bf16_decode(uint16_t h)
+{
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* fp32 -> bf16, round to nearest even. */
+uint16_t moe_ref_bf16_encode(float x)
+{
+    uint32_t u;
+    memcpy(&u, &x, 4);
+    if (isnan(x))
+        return (uint16_t)((u >> 16) | 0x0040);
+    u += 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Routing (stage 1 of the Fused MoE paragraph)                              */
+/* ------------------------------------------------------------------------ */
+
+/* A fully specified fp32 exponential.  Routing indices are compared bit for
+ * bit, so the exponential is fixed operation by operation instead of being
+ * left to a maths library: clamp, split x = n ln2 + r with a two-part ln2,
+ * degree-7 Taylor polynomial in r by Horner with fused multiply-adds, scale
+ * by 2^n through the exponent field. */
+float moe_ref_expdet(float x)
+{
+    float n, r, p, two_n;
+    uint32_t bits;
+    x = fminf(fmaxf(x, -87.0f), 88.0f);
+    n = nearbyintf(x * 0x1.715476p+0f);     /* log2(e) rounded to fp32 */
+    r = fmaf(n, -0x1.62e4p-1f, x);          /* ln2, high part (few bits) */
+    r = fmaf(n, -0x1.7f7d1cp-20f, r);       /* ln2, low part */
+    p = 0x1.a01a02p-13f;                    /* 1/5040 */
+    p = fmaf(p, r, 0x1.6c16c2p-10f);        /* 1/720 */
+    p = fmaf(p, r, 0x1.111112p-7f);         /* 1/120 */
+    p = fmaf(p, r, 0x1.555556p-5f);         /* 1/24 */
+    p = fmaf(p, r, 0x1.555556p-3f);         /* 1/6 */
+    p = fmaf(p, r, 0.5f);
+    p = fmaf(p, r, 1.0f);
+    p = fmaf(p, r, 1.0f);
+    bits = (uint32_t)((int)n + 127) << 23;
+    memcpy(&two_n, &bits, 4);
+    return p * two_n;
+}
+
+float moe_ref_sigmoid(float x)
+{
+    return 1.0f / (1.0f + moe_ref_expdet(-x));
+}
+
+/* Grouped routing of DeepSeek-V3 as the paper's stage 1 lists it (sigmoid,
+ * group-wise top-2, final top-K), with the reading that the group-wise top-2
+ * scores a group, the KG best groups are kept, and the K best experts of the
+ * kept groups are selected.
+ *
+ *   logits [T,E] fp32, bias [E] bf16 bits.
+ *   topk_idx [T,K] int32, topk_w [T,K] fp32: order = descending biased score,
+ *   ties by ascending expert index.
+ *   sig_out (optional) [T,E] the unbiased sigmoid scores. */
+int moe_ref_route(int T, int E, int G, int KG, int K, const float *logits,
+                  const uint16_t *bias_bf16, float scaling, int32_t *topk_idx,
+                  float *topk_w, float *sig_out)
+{
+    int per, t, e, g, j;
+    float *sig, *b, *gs;
+    unsigned char *group_kept, *taken;
+    if (T < 0 || E <= 0 || G <= 0 || E % G != 0 || KG <= 0 || KG > G || K <= 0)
+        return MOE_REF_BAD_ARG;
+    per = E / G;
+    if (per < 2 || K > KG * per)
+        return MOE_REF_BAD_ARG;
+    sig = (float *)malloc(sizeof(float) * E);
+    b = (float *)malloc(sizeof(float) * E);
+    gs = (float *)malloc(sizeof(float) * G);
+    group_kept = (unsigned char *)malloc(G);
+    taken = (unsigned char *)malloc(E);
+    if (!sig || !b || !gs || !group_kept || !taken)
+        return MOE_REF_NO_MEM;
+
+    for (t = 0; t < T; ++t) {
+        float den;
+        /* scores */
+        for (e = 0; e < E; ++e) {
+            sig[e] = moe_ref_sigmoid(logits[(size_t)t * E + e]);
+            b[e] = sig[e] + moe_ref_bf16_decode(bias_bf16[e]);
+            if (sig_out)
+                sig_out[(size_t)t * E + e] = sig[e];
+        }
+        /* group score = largest + second largest biased score of the group */
+        for (g = 0; g < G; ++g) {
+            int i1 = -1, i2 = -1;
+            for (e = g * per; e < (g + 1) * per; ++e)
+                if (i1 < 0 || b[e] > b[i1])
+                    i1 = e;
+            for (e = g * per; e < (g + 1) * per; ++e)
+                if (e != i1 && (i2 < 0 || b[e] > b[i2]))
+                    i2 = e;
+            gs[g] = b[i1] + b[i2];
+        }
+        /* keep the KG best groups, ties to the smaller group index */
+        memset(group_kept, 0, G);
+        for (j = 0; j < KG; ++j) {
+            int best = -1;
+            for (g = 0; g < G; ++g)
+                if (!group_kept[g] && (best < 0 || gs[g] > gs[best]))
+                    best = g;
+            group_kept[best] = 1;
+        }
+        /* select the K best experts of the kept groups, ties to the smaller
+         * expert index; the selection order is the canonical output order */
+        memset(taken, 0, E);
+        for (j = 0; j < K; ++j) {
+            int best = -1;
+            for (e = 0; e < E; ++e)
+                if (group_kept[e / per] && !taken[e] &&
+                    (best < 0 || b[e] > b[best]))
+                    best = e;
+            taken[best] = 1;
+            topk_idx[(size_t)t * K + j] = best;
+        }
+        /* weights: unbiased scores renormalised over the K selected, then
+         * multiplied by the routed scaling factor */
+        den = 0.0f;
+        for (j = 0; j < K; ++j)
+            den = den + sig[topk_idx[(size_t)t * K + j]];
+        for (j = 0; j < K; ++j)
+            topk_w[(size_t)t * K + j] =
+                (sig[topk_idx[(size_t)t * K + j]] / den) * scaling;
+    }
+    free(sig);
+    free(b);
+    free(gs);
+    free(group_kept);
+    free(taken);
+    return MOE_REF_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Histogram and canonical permutation (stage 2)                             */
+/* ------------------------------------------------------------------------ */
+
+/* Slot id = t*K + j.  A slot is local iff off <= expert < off + E_loc.
+ * Rows are ordered by local expert, and within an expert by ascending token.
+ *   count[E_loc], offset[E_loc+1] (exclusive scan), row_to_slot[T*K] (first
+ *   S entries valid, rest -1), slot_to_row[T*K] (-1 for dropped slots).
+ * Returns S (>= 0) or a negative error. */
+int moe_ref_permute(int T, int K, const int32_t *topk_idx, int off, int E_loc,
+                    int32_t *count, int32_t *offset, int32_t *row_to_slot,
+                    int32_t *slot_to_row)
+{
+    int e, t, j, row = 0;
+    if (T < 0 || K <= 0 || E_loc <= 0)
+        return MOE_REF_BAD_ARG;
+    for (t = 0; t < T * K; ++t) {
+        row_to_slot[t] = -1;
+        slot_to_row[t] = -1;
+    }
+    for (e = 0; e < E_loc; ++e) {
+        offset[e] = row;
+        for (t = 0; t < T; ++t)
+            for (j = 0; j < K; ++j)
+                if (topk_idx[(size_t)t * K + j] == off + e) {
+                    row_to_slot[row] = t * K + j;
+                    slot_to_row[t * K + j] = row;
+                    ++row;
+                }
+        count[e] = row - offset[e];
+    }
+    offset[E_loc] = row;
+    return row;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Expert MLP on one row (stages 3: GEMM1, SwiGLU, re-quantisation, GEMM2)   */
+/* ------------------------------------------------------------------------ */
+
+/* Sum of 128 exact fp32 products with 16 interleaved partial sums combined in
+ * a fixed binary tree (fp32), or one fp64 running sum. */
+static float block_dot(const float *a, const float *w, int use_double)
+{
+    int i, l;
+    if (use_double) {
+        double s = 0.0;
+        for (i = 0; i < QBLOCK; ++i)
+            s += (double)a[i] * (double)w[i];
+        return (float)s;
+    } else {
+        float lane[16];
+        for (l = 0; l < 16; ++l)
+            lane[l] = 0.0f;
+        for (i = 0; i < QBLOCK; i += 16)
+            for (l = 0; l < 16; ++l)
+                lane[l] = lane[l] + a[i + l] * w[i + l];
+        for (l = 0; l < 8; ++l)
+            lane[l] = lane[l] + lane[l + 8];
+        for (l = 0; l < 4; ++l)
+            lane[l] = lane[l] + lane[l + 4];
+        for (l = 0; l < 2; ++l)
+            lane[l] = lane[l] + lane[l + 2];
+        return lane[0] + lane[1];
+    }
+}
+
+/* out[n] = sum over K-blocks kb of (x_s[kb] * w_s[n/128][kb]) * dot_kb, for a
+ * weight matrix w_q [N, Kdim] (Kdim contiguous) with scales
+ * w_s [N/128, Kdim/128]; xd is the row already decoded to fp32 (the codes,
+ * not yet multiplied by their scales). */
+static void blockscaled_matvec(int N, int Kdim, const float *xd,
+                               const float *x_s, const uint8_t *w_q,
+                               const float *w_s, const float *lut,
+                               int use_double, float *wrow, float *out)
+{
+    int n, k, kb, nkb = Kdim / QBLOCK;
+    for (n = 0; n < N; ++n) {
+        const uint8_t *wr = w_q + (size_t)n * Kdim;
+        float acc = 0.0f;
+        double accd = 0.0;
+        for (k = 0; k < Kdim; ++k)
+            wrow[k] = lut[wr[k]];
+        for (kb = 0; kb < nkb; ++kb) {
+            float p = block_dot(xd + kb * QBLOCK, wrow + kb * QBLOCK, use_double);
+            float sc = x_s[kb] * w_s[(size_t)(n / QBLOCK) * nkb + kb];
+            if (use_double)
+                accd += (double)sc * (double)p;
+            else
+                acc = acc + sc * p;
+        }
+        out[n] = use_double ? (float)accd : acc;
+    }
+}
+
+/* One (token, expert) slot.
+ *   x_q [H] e4m3 codes, x_s [H/128]; w13 [2I,H] codes, w13_s [2I/128,H/128];
+ *   w2 [H,I] codes, w2_s [H/128,I/128].
+ *   gate_first != 0: rows [0,I) of w13 are the gate (SiLU side), rows [I,2I)
+ *   the up projection; 0 swaps the halves.
+ *   y [H] fp32 result; c_q [I] / c_s [I/128] (optional) the re-quantised
+ *   SwiGLU output that feeds GEMM2. */
+int moe_ref_mlp_row(int H, int I, const uint8_t *x_q, const float *x_s,
+                    const uint8_t *w13, const float *w13_s, const uint8_t *w2,
+                    const float *w2_s, int gate_first, int use_double, float *y,
+                    uint8_t *c_q, float *c_s)
+{
+    float lut[256];
+    float *xd, *wrow, *h13, *c, *cd, *cs;
+    int i, k, jb, maxdim = H > I ? H : I;
+    if (H <= 0 || I <= 0 || H % QBLOCK || I % QBLOCK)
+        return MOE_REF_BAD_ARG;
+    for (i = 0; i < 256; ++i)
+        lut[i] = moe_ref_e4m3_decode((uint8_t)i);
+    xd = (float *)malloc(sizeof(float) * H);
+    wrow = (float *)malloc(sizeof(float) * maxdim);
+    h13 = (float *)malloc(sizeof(float) * 2 * I);
+    c = (float *)malloc(sizeof(float) * I);
+    cd = (float *)malloc(sizeof(float) * I);
+    cs = (float *)malloc(sizeof(float) * (I / QBLOCK));
+    if (!xd || !wrow || !h13 || !c || !cd || !cs)
+        return MOE_REF_NO_MEM;
+
+    /* GEMM1: [H] -> [2I] */
+    for (k = 0; k < H; ++k)
+        xd[k] = lut[x_q[k]];
+    blockscaled_matvec(2 * I, H, xd, x_s, w13, w13_s, lut, use_double, wrow, h13);
+
+    /* SwiGLU: silu(gate) * up */
+    for (i = 0; i < I; ++i) {
+        float g = gate_first ? h13[i] : h13[I + i];
+        float u = gate_first ? h13[I + i] : h13[i];
+        c[i] = (g / (1.0f + expf(-g))) * u;
+    }
+
+    /* re-quantisation: per 128 columns, scale = amax / 448 (1 if the block is
+     * all zero), code = e4m3(c / scale) */
+    for (jb = 0; jb < I / QBLOCK; ++jb) {
+        float amax = 0.0f, sc;
+        for (i = jb * QBLOCK; i < (jb + 1) * QBLOCK; ++i)
+            amax = fmaxf(amax, fabsf(c[i]));
+        sc = (amax == 0.0f) ? 1.0f : amax / 448.0f;
+        cs[jb] = sc;
+        for (i = jb * QBLOCK; i < (jb + 1) * QBLOCK; ++i) {
+            uint8_t q = moe_ref_e4m3_encode(c[i] / sc);
+            cd[i] = lut[q];
+            if (c_q)
+                c_q[i] = q;
+        }
+        if (c_s)
+            c_s[jb] = sc;
+    }
+
+    /* GEMM2: [I] -> [H] */
+    blockscaled_matvec(H, I, cd, cs, w2, w2_s, lut, use_double, wrow, y);
+
+    free(xd);
+    free(wrow);
+    free(h13);
+    free(c);
+    free(cd);
+    free(cs);
+    return MOE_REF_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Whole forward                                                              */
+/* ------------------------------------------------------------------------ */
+
+/* All arrays are host arrays.
+ *   hidden_q [T,H] e4m3 codes; hidden_s [T,H/128] fp32 (or [H/128,T] when
+ *   scale_layout == 1); logits [T,E]; bias [E] bf16 bits;
+ *   w13 [E_loc,2I,H]; w13_s [E_loc,2I/128,H/128]; w2 [E_loc,H,I];
+ *   w2_s [E_loc,H/128,I/128].
+ *   tokens: NULL -> every token, out is [T,H]; otherwise a list of n_tokens
+ *   token ids and out is [n_tokens,H] (row i belongs to tokens[i]).
+ *   out: bf16 bits.  topk_idx/topk_w (optional) [T,K] for every token. */
+int moe_ref_forward(int T, int H, int I, int E, int E_loc, int G, int KG, int K,
+                    int scale_layout, int gate_first, int use_double,
+                    const uint8_t *hidden_q, const float *hidden_s,
+                    const float *logits, const uint16_t *bias,
+                    const uint8_t *w13, const float *w13_s, const uint8_t *w2,
+                    const float *w2_s, int off, float scaling,
+                    const int32_t *tokens, int n_tokens, uint16_t *out,
+                    int32_t *topk_idx, float *topk_w)
+{
+    int rc, i, j, h, kb, nT = tokens ? n_tokens : T, nkb;
+    int32_t *idx;
+    float *w, *xs, *y, *acc;
+    if (T < 0 || H <= 0 || I <= 0 || H % QBLOCK || I % QBLOCK || E_loc <= 0 ||
+        off < 0 || off + E_loc > E || K <= 0)
+        return MOE_REF_BAD_ARG;
+    nkb = H / QBLOCK;
+    idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(T > 0 ? T : 1) * K);
+    w = (float *)malloc(sizeof(float) * (size_t)(T > 0 ? T : 1) * K);
+    xs = (float *)malloc(sizeof(float) * nkb);
+    y = (float *)malloc(sizeof(float) * H);
+    acc = (float *)malloc(sizeof(float) * H);
+    if (!idx || !w || !xs || !y || !acc)
+        return MOE_REF_NO_MEM;
+    rc = moe_ref_route(T, E, G, KG, K, logits, bias, scaling, idx, w, NULL);
+    if (rc != MOE_REF_OK)
+        return rc;
+    if (topk_idx)
+        memcpy(topk_idx, idx, sizeof(int32_t) * (size_t)T * K);
+    if (topk_w)
+        memcpy(topk_w, w, sizeof(float) * (size_t)T * K);
+
+    for (i = 0; i < nT; ++i) {
+        int t = tokens ? tokens[i] : i;
+        if (t < 0 || t >= T)
+            return MOE_REF_BAD_ARG;
+        for (kb = 0; kb < nkb; ++kb)
+            xs[kb] = scale_layout ? hidden_s[(size_t)kb * T + t]
+                                  : hidden_s[(size_t)t * nkb + kb];
+        for (h = 0; h < H; ++h)
+            acc[h] = 0.0f;
+        /* combine: the token's local slots in canonical order, fp32 */
+        for (j = 0; j < K; ++j) {
+            int e = idx[(size_t)t * K + j] - off;
+            if (e < 0 || e >= E_loc)
+                continue; /* non-local route: dropped */
+            rc = moe_ref_mlp_row(
+                H, I, hidden_q + (size_t)t * H, xs,
+                w13 + (size_t)e * 2 * I * H,
+                w13_s + (size_t)e * (2 * I / QBLOCK) * (H / QBLOCK),
+                w2 + (size_t)e * H * I,
+                w2_s + (size_t)e * (H / QBLOCK) * (I / QBLOCK), gate_first,
+                use_double, y, NULL, NULL);
+            if (rc != MOE_REF_OK)
+                return rc;
+            for (h = 0; h < H; ++h)
+                acc[h] = acc[h] + w[(size_t)t * K + j] * y[h];
+        }
+        for (h = 0; h < H; ++h)
+            out[(size_t)i * H + h] = moe_ref_bf16_encode(acc[h]);
+    }
+    free(idx);
+    free(w);
+    free(xs);
+    free(y);
+    free(acc);
+    return MOE_REF_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Dense brute force: every local expert for every token, weight 0 when the  */
+/* expert was not selected.  Written separately from moe_ref_forward and     */
+/* moe_ref_mlp_row (plain triple loops, fp64 sums) for tiny problems only.   */
+/* ------------------------------------------------------------------------ */
+int moe_ref_dense_bruteforce(int T, int H, int I, int E, int E_loc, int G,
+                             int KG, int K, int gate_first,
+                             const uint8_t *hidden_q, const float *hidden_s,
+                             const float *logits, const uint16_t *bias,
+                             const uint8_t *w13, const float *w13_s,
+                             const uint8_t *w2, const float *w2_s, int off,
+                             float scaling, float *out_f32)
+{
+    int t, e, j, n, k, h, rc;
+    int nkbH = H / QBLOCK, nkbI = I / QBLOCK;
+    int32_t *idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(T + 1) * K);
+    float *wk = (float *)malloc(sizeof(float) * (size_t)(T + 1) * K);
+    double *h13 = (double *)malloc(sizeof(double) * 2 * I);
+    float *c = (float *)malloc(sizeof(float) * I);
+    float *cdq = (float *)malloc(sizeof(float) * I);
+    if (!idx || !wk || !h13 || !c || !cdq)
+        return MOE_REF_NO_MEM;
+    rc = moe_ref_route(T, E, G, KG, K, logits, bias, scaling, idx, wk, NULL);
+    if (rc != MOE_REF_OK)
+        return rc;
+    for (t = 0; t < T; ++t) {
+        for (h = 0; h < H; ++h)
+            out_f32[(size_t)t * H + h] = 0.0f;
+        for (e = 0; e < E_loc; ++e) {
+            const uint8_t *W13 = w13 + (size_t)e * 2 * I * H;
+            const float *S13 = w13_s + (size_t)e * (2 * I / QBLOCK) * nkbH;
+            const uint8_t *W2 = w2 + (size_t)e * H * I;
+            const float *S2 = w2_s + (size_t)e * nkbH * nkbI;
+            float dense_w = 0.0f;
+            for (j = 0; j < K; ++j)
+                if (idx[(size_t)t * K + j] == off + e)
+                    dense_w = wk[(size_t)t * K + j];
+            for (n = 0; n < 2 * I; ++n) {
+                double s = 0.0;
+                for (k = 0; k < H; ++k)
+                    s += (double)moe_ref_e4m3_decode(hidden_q[(size_t)t * H + k]) *
+                         (double)hidden_s[(size_t)t * nkbH + k / QBLOCK] *
+                         (double)moe_ref_e4m3_decode(W13[(size_t)n * H + k]) *
+                         (double)S13[(size_t)(n / QBLOCK) * nkbH + k / QBLOCK];
+                h13[n] = s;
+            }
+            for (n = 0; n < I; ++n) {
+                float g = (float)(gate_first ? h13[n] : h13[I + n]);
+                float u = (float)(gate_first ? h13[I + n] : h13[n]);
+                c[n] = (g / (1.0f + expf(-g))) * u;
+            }
+            for (n = 0; n < I; n += QBLOCK) {
+                float amax = 0.0f, sc;
+                for (k = n; k < n + QBLOCK; ++k)
+                    amax = fmaxf(amax, fabsf(c[k]));
+                sc = amax == 0.0f ? 1.0f : amax / 448.0f;
+                for (k = n; k < n + QBLOCK; ++k)
+                    cdq[k] = moe_ref_e4m3_decode(moe_ref_e4m3_encode(c[k] / sc)) * sc;
+            }
+            for (h = 0; h < H; ++h) {
+                double s = 0.0;
+                for (k = 0; k < I; ++k)
+                    s += (double)cdq[k] *
+                         (double)moe_ref_e4m3_decode(W2[(size_t)h * I + k]) *
+                         (double)S2[(size_t)(h / QBLOCK) * nkbI + k / QBLOCK];
+                out_f32[(size_t)t * H + h] += dense_w * (float)s;
+            }
+        }
+    }
+    free(idx);
+    free(wk);
+    free(h13);
+    free(c);
+    free(cdq);
+    return MOE_REF_OK;
+}
