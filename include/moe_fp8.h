@@ -1,0 +1,138 @@
+/*
+ * moe_fp8.h -- C ABI of the B200 (sm_100a) fused block-scaled FP8 MoE forward.
+ *
+ * The operation is the "Fused MoE" workload of the paper (Section "Kernel
+ * Design and Optimization", subsection "Fused MoE"): the DeepSeek-V3 MoE block
+ * in four stages -- (1) routing: sigmoid scores, group-wise top-2 over 8
+ * groups, final top-K = 8; (2) gathering the active rows of each expert into a
+ * contiguous FP8 layout with 128-element fp32 block scales; (3) the gated MLP:
+ * FP8 block-scaled GEMM1 [T,7168]->[T,4096], SwiGLU, re-quantisation, FP8
+ * block-scaled GEMM2 [T,2048]->[T,7168]; (4) scattering the expert outputs
+ * back to token positions weighted by the routing scores.  As in the paper's
+ * final implementation, all metadata is built on the GPU and the hot path never
+ * synchronises the stream.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its comment says "host".
+ *   - The library never allocates, frees or retains caller tensors; scratch
+ *     memory is one caller-owned workspace (moe_fp8_set_workspace).
+ *   - Functions return 0 on success and a negative MOE_FP8_ERR_* otherwise; on
+ *     error nothing has been enqueued.  There is no CPU fallback: without a
+ *     compute-capability 10.x device moe_fp8_create fails.
+ *   - moe_fp8_forward only enqueues work on `stream` and returns; faults found
+ *     on the device (a bounded wait that gave up, an out-of-range row) are
+ *     recorded in a status word readable through moe_fp8_debug_export.
+ *   - One handle serves one stream at a time.  Weights are treated as
+ *     immutable while the same weight pointers are passed (their TMA
+ *     descriptors are cached per pointer pair); nothing is cached on
+ *     activations, logits or outputs.
+ *   - Inputs must be finite.  Base addresses must be 16-byte aligned.
+ */
+#ifndef MOE_FP8_H_
+#define MOE_FP8_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOE_FP8_OK 0
+#define MOE_FP8_ERR_BAD_ARG (-1)          /* null/misaligned pointer, T out of range, offset out of range */
+#define MOE_FP8_ERR_UNSUPPORTED_DIMS (-2) /* layer shape outside what the kernels are built for */
+#define MOE_FP8_ERR_NO_WORKSPACE (-3)     /* workspace missing or too small */
+#define MOE_FP8_ERR_CUDA (-4)             /* a CUDA call failed; see moe_fp8_last_cuda_error */
+#define MOE_FP8_ERR_ARCH (-5)             /* current device is not compute capability 10.x */
+
+/* Layer shape, fixed at creation.  Supported: num_experts = 256, n_group = 8,
+ * topk_group = 4, top_k = 8 (the DeepSeek-V3 routing of stage 1); hidden a
+ * multiple of 256, intermediate a multiple of 128; 1 <= num_local_experts <= 256. */
+typedef struct moe_fp8_config {
+    int hidden;              /* H, 7168 */
+    int intermediate;        /* I, 2048 */
+    int num_experts;         /* E, 256 global experts */
+    int num_local_experts;   /* E_loc, experts whose weights live on this GPU */
+    int n_group;             /* 8 */
+    int topk_group;          /* 4 */
+    int top_k;               /* 8 */
+    int max_tokens;          /* upper bound on T; sizes the workspace */
+    int hidden_scale_layout; /* 0: hidden_scale is [T, H/128]; 1: [H/128, T] */
+    int gate_first;          /* 1: w13 rows [0,I) are the gate (SiLU side), [I,2I) the up projection; 0: swapped */
+} moe_fp8_config;
+
+typedef struct moe_fp8_handle_s* moe_fp8_handle_t;
+
+/* Host only.  Validates the shape, then requires a cc 10.x current device. */
+int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out);
+int moe_fp8_destroy(moe_fp8_handle_t h);
+
+/* Bytes of device scratch needed for cfg.max_tokens tokens. */
+size_t moe_fp8_workspace_bytes(moe_fp8_handle_t h);
+/* Hands the library a caller-owned device buffer (1024-byte aligned) that must
+ * stay valid until it is replaced or the handle destroyed. */
+int moe_fp8_set_workspace(moe_fp8_handle_t h, void* dev_workspace, size_t bytes);
+
+/*
+ * One forward pass of the layer for T tokens (stages 1-4 above), enqueued on
+ * `stream` (a cudaStream_t).  T = 0 is valid and enqueues nothing.
+ *
+ *   hidden_fp8     e4m3 [T, H]            activations
+ *   hidden_scale   fp32 [T, H/128]        one scale per token per 128 columns
+ *   router_logits  fp32 [T, 256]
+ *   routing_bias   bf16 [256]             added to the sigmoid score for selection only
+ *   w13            e4m3 [E_loc, 2I, H]    gate and up projections, H contiguous
+ *   w13_scale      fp32 [E_loc, 2I/128, H/128]
+ *   w2             e4m3 [E_loc, H, I]     down projection, I contiguous
+ *   w2_scale       fp32 [E_loc, H/128, I/128]
+ *   local_expert_offset  first global expert id held locally; routes to experts
+ *                        outside [offset, offset+E_loc) are dropped after the
+ *                        weights were normalised over all 8 selected experts
+ *   scaling_factor routed scaling factor (2.5)
+ *   out            bf16 [T, H], fully overwritten (zeros for tokens without a local expert)
+ */
+int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const float* hidden_scale,
+                    const float* router_logits, const void* routing_bias, const void* w13,
+                    const float* w13_scale, const void* w2, const float* w2_scale, int local_expert_offset,
+                    float scaling_factor, void* out, void* stream);
+
+/*
+ * The same pass for callers whose per-step tensors live in HOST memory
+ * (preferably pinned): copies hidden_fp8, hidden_scale and router_logits to
+ * staging areas inside the workspace, runs moe_fp8_forward, copies `out` back
+ * and waits for the stream.  Weights, their scales and the bias stay device
+ * pointers.  host_* arguments are host pointers with the layouts above.
+ */
+int moe_fp8_forward_host(moe_fp8_handle_t h, int T, const void* host_hidden_fp8, const float* host_hidden_scale,
+                         const float* host_router_logits, const void* routing_bias, const void* w13,
+                         const float* w13_scale, const void* w2, const float* w2_scale, int local_expert_offset,
+                         float scaling_factor, void* host_out, void* stream);
+
+/*
+ * Test hook: copies internal results of the LAST forward on this handle into
+ * caller buffers (device pointers, any may be NULL), enqueued on `stream`.
+ *   topk_idx       int32 [T, 8]  selected experts, descending biased score
+ *   topk_w         fp32  [T, 8]
+ *   expert_count   int32 [E_loc]
+ *   expert_offset  int32 [E_loc+1]   exclusive scan of the counts
+ *   row_to_slot    int32 [T*8]       row -> slot id t*8+j (experts ascending,
+ *                                    tokens ascending inside an expert); first S valid
+ *   a2_fp8         e4m3  [T*8, I]    re-quantised SwiGLU output per row (first S rows)
+ *   a2_scale       fp32  [T*8, I/128]
+ *   y_rows         bf16  [T*8, H]    GEMM2 output per row before the combine
+ *   status_word    int32 [1]         0, or the first device-side fault code
+ */
+int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w, int* expert_count,
+                         int* expert_offset, int* row_to_slot, void* a2_fp8, float* a2_scale, void* y_rows,
+                         int* status_word, void* stream);
+
+/* CUDA error code (cudaError_t as int) of the last MOE_FP8_ERR_CUDA on this handle. */
+int moe_fp8_last_cuda_error(moe_fp8_handle_t h);
+/* Kernel launches enqueued by the last moe_fp8_forward on this handle. */
+int moe_fp8_last_launch_count(moe_fp8_handle_t h);
+/* Static string for a return code. */
+const char* moe_fp8_strerror(int rc);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_FP8_H_ */

@@ -1,0 +1,170 @@
+"""ctypes binding of include/moe_fp8.h.  Argument marshalling only: every step
+of the forward pass runs in the CUDA library.  PyTorch supplies device memory
+and streams."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from .build import LIB_PATH
+
+OK = 0
+ERR_BAD_ARG, ERR_UNSUPPORTED_DIMS, ERR_NO_WORKSPACE, ERR_CUDA, ERR_ARCH = -1, -2, -3, -4, -5
+
+EXPORTS = (
+    "moe_fp8_create", "moe_fp8_destroy", "moe_fp8_workspace_bytes", "moe_fp8_set_workspace", "moe_fp8_forward",
+    "moe_fp8_forward_host", "moe_fp8_debug_export", "moe_fp8_last_cuda_error", "moe_fp8_last_launch_count",
+    "moe_fp8_strerror",
+)
+
+
+class Config(C.Structure):
+    _fields_ = [(n, C.c_int) for n in (
+        "hidden", "intermediate", "num_experts", "num_local_experts", "n_group", "topk_group", "top_k",
+        "max_tokens", "hidden_scale_layout", "gate_first")]
+
+
+class MoeFp8Error(RuntimeError):
+    def __init__(self, rc: int, msg: str):
+        super().__init__(f"moe_fp8 error {rc}: {msg}")
+        self.rc = rc
+
+
+_lib = None
+
+
+def load_library() -> C.CDLL:
+    """Loads the CUDA library; raises if it has not been built (no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise MoeFp8Error(ERR_CUDA, f"{LIB_PATH} is missing: run `python -m paper_2608_14560_b200.build` "
+                                        "(there is no CPU or PyTorch fallback)")
+        lib = C.CDLL(LIB_PATH)
+        vp, ip, fp = C.c_void_p, C.c_void_p, C.c_void_p
+        lib.moe_fp8_create.argtypes = [C.POINTER(Config), C.POINTER(C.c_void_p)]
+        lib.moe_fp8_create.restype = C.c_int
+        lib.moe_fp8_destroy.argtypes = [vp]
+        lib.moe_fp8_destroy.restype = C.c_int
+        lib.moe_fp8_workspace_bytes.argtypes = [vp]
+        lib.moe_fp8_workspace_bytes.restype = C.c_size_t
+        lib.moe_fp8_set_workspace.argtypes = [vp, vp, C.c_size_t]
+        lib.moe_fp8_set_workspace.restype = C.c_int
+        fwd = [vp, C.c_int, vp, fp, fp, vp, vp, fp, vp, fp, C.c_int, C.c_float, vp, vp]
+        lib.moe_fp8_forward.argtypes = fwd
+        lib.moe_fp8_forward.restype = C.c_int
+        lib.moe_fp8_forward_host.argtypes = fwd
+        lib.moe_fp8_forward_host.restype = C.c_int
+        lib.moe_fp8_debug_export.argtypes = [vp, C.c_int, ip, fp, ip, ip, ip, vp, fp, vp, ip, vp]
+        lib.moe_fp8_debug_export.restype = C.c_int
+        lib.moe_fp8_last_cuda_error.argtypes = [vp]
+        lib.moe_fp8_last_cuda_error.restype = C.c_int
+        lib.moe_fp8_last_launch_count.argtypes = [vp]
+        lib.moe_fp8_last_launch_count.restype = C.c_int
+        lib.moe_fp8_strerror.argtypes = [C.c_int]
+        lib.moe_fp8_strerror.restype = C.c_char_p
+        _lib = lib
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+class MoeFp8:
+    """One layer shape + its workspace.  Same names as the C entry points."""
+
+    def __init__(self, hidden=7168, intermediate=2048, num_experts=256, num_local_experts=32, n_group=8,
+                 topk_group=4, top_k=8, max_tokens=1024, hidden_scale_layout=0, gate_first=True,
+                 device="cuda:0"):
+        self.lib = load_library()
+        self.cfg = Config(hidden, intermediate, num_experts, num_local_experts, n_group, topk_group, top_k,
+                          max_tokens, hidden_scale_layout, int(gate_first))
+        self.device = torch.device(device)
+        self.handle = C.c_void_p()
+        if self.device.type == "cuda":
+            torch.cuda.set_device(self.device)
+        self._check(self.lib.moe_fp8_create(C.byref(self.cfg), C.byref(self.handle)))
+        self.workspace_bytes = int(self.lib.moe_fp8_workspace_bytes(self.handle))
+        self.workspace = torch.empty(self.workspace_bytes + 1024, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        self._ws_ptr = (base + 1023) // 1024 * 1024
+        self._check(self.lib.moe_fp8_set_workspace(self.handle, C.c_void_p(self._ws_ptr), self.workspace_bytes))
+
+    def _check(self, rc: int):
+        if rc != OK:
+            msg = self.lib.moe_fp8_strerror(rc).decode()
+            if rc == ERR_CUDA and self.handle:
+                msg += f" (cudaError {self.lib.moe_fp8_last_cuda_error(self.handle)})"
+            raise MoeFp8Error(rc, msg)
+
+    def close(self):
+        if self.handle:
+            self.lib.moe_fp8_destroy(self.handle)
+            self.handle = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _stream(self, stream):
+        s = torch.cuda.current_stream(self.device) if stream is None else stream
+        return C.c_void_p(s.cuda_stream)
+
+    def forward(self, inp: dict, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+        """moe_fp8_forward on device tensors (dict keys as synthetic.make_inputs)."""
+        T = inp["router_logits"].shape[0]
+        if out is None:
+            out = torch.empty(T, self.cfg.hidden, dtype=torch.bfloat16, device=self.device)
+        self._check(self.lib.moe_fp8_forward(
+            self.handle, T, _ptr(inp["hidden_fp8"]), _ptr(inp["hidden_scale"]), _ptr(inp["router_logits"]),
+            _ptr(inp["routing_bias"]), _ptr(inp["w13"]), _ptr(inp["w13_scale"]), _ptr(inp["w2"]),
+            _ptr(inp["w2_scale"]), int(inp["local_expert_offset"]), float(inp["scaling_factor"]), _ptr(out),
+            self._stream(stream)))
+        return out
+
+    def forward_host(self, host_act: dict, weights: dict, host_out: torch.Tensor, stream=None) -> torch.Tensor:
+        """moe_fp8_forward_host: hidden_fp8 / hidden_scale / router_logits / out in (pinned) host memory."""
+        T = host_act["router_logits"].shape[0]
+        self._check(self.lib.moe_fp8_forward_host(
+            self.handle, T, _ptr(host_act["hidden_fp8"]), _ptr(host_act["hidden_scale"]),
+            _ptr(host_act["router_logits"]), _ptr(weights["routing_bias"]), _ptr(weights["w13"]),
+            _ptr(weights["w13_scale"]), _ptr(weights["w2"]), _ptr(weights["w2_scale"]),
+            int(weights["local_expert_offset"]), float(weights["scaling_factor"]), _ptr(host_out),
+            self._stream(stream)))
+        return host_out
+
+    def last_launch_count(self) -> int:
+        return int(self.lib.moe_fp8_last_launch_count(self.handle))
+
+    def debug_export(self, T: int, rows: bool = True, stream=None) -> dict:
+        """moe_fp8_debug_export -> dict of device tensors (see the header for shapes)."""
+        dev, EL = self.device, self.cfg.num_local_experts
+        I, H = self.cfg.intermediate, self.cfg.hidden
+        r = {
+            "topk_idx": torch.empty(T, 8, dtype=torch.int32, device=dev),
+            "topk_w": torch.empty(T, 8, dtype=torch.float32, device=dev),
+            "expert_count": torch.empty(EL, dtype=torch.int32, device=dev),
+            "expert_offset": torch.empty(EL + 1, dtype=torch.int32, device=dev),
+            "row_to_slot": torch.full((T * 8,), -1, dtype=torch.int32, device=dev),
+            "status": torch.zeros(1, dtype=torch.int32, device=dev),
+        }
+        if rows:
+            r["a2_fp8"] = torch.zeros(T * 8, I, dtype=torch.uint8, device=dev)
+            r["a2_scale"] = torch.zeros(T * 8, I // 128, dtype=torch.float32, device=dev)
+            r["y_rows"] = torch.zeros(T * 8, H, dtype=torch.bfloat16, device=dev)
+        self._check(self.lib.moe_fp8_debug_export(
+            self.handle, T, _ptr(r["topk_idx"]), _ptr(r["topk_w"]), _ptr(r["expert_count"]),
+            _ptr(r["expert_offset"]), _ptr(r["row_to_slot"]), _ptr(r.get("a2_fp8")), _ptr(r.get("a2_scale")),
+            _ptr(r.get("y_rows")), _ptr(r["status"]), self._stream(stream)))
+        return r
+
+    def status(self) -> int:
+        s = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self._check(self.lib.moe_fp8_debug_export(self.handle, 0, None, None, None, None, None, None, None, None,
+                                                  _ptr(s), self._stream(None)))
+        return int(s.item())

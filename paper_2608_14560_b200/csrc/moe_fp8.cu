@@ -1,0 +1,419 @@
+// Host side of the C ABI declared in include/moe_fp8.h: handle, workspace
+// carving, TMA descriptors and the launch sequence of one forward pass.
+#include "../../include/moe_fp8.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "ptx.cuh"
+#include "routing.cuh"
+#include "permute.cuh"
+#include "gemm.cuh"
+#include "combine.cuh"
+
+namespace {
+
+using namespace moe;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr size_t WS_ALIGN = 1024;
+inline size_t align_up(size_t x, size_t a = WS_ALIGN) { return (x + a - 1) / a * a; }
+
+struct WsLayout {
+    size_t topk_idx, topk_w, block_hist, expert_count, expert_offset, padded_offset, tile_expert, tile_rows,
+        num_m_tiles, slot_to_row, row_to_slot, row_token, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
+        stage_scale, stage_logits, stage_out, total;
+    int row_cap, max_m_tiles, max_blocks;
+};
+
+WsLayout make_layout(const moe_fp8_config& c) {
+    WsLayout L;
+    const size_t Tm = static_cast<size_t>(c.max_tokens > 0 ? c.max_tokens : 1);
+    const size_t slots = Tm * 8;
+    size_t pad_experts = static_cast<size_t>(c.num_local_experts) < slots ? c.num_local_experts : slots;
+    L.row_cap = static_cast<int>(align_up(slots + pad_experts * (TILE_M - 1), TILE_M));
+    L.max_m_tiles = L.row_cap / TILE_M;
+    L.max_blocks = static_cast<int>((Tm + P_TOKENS_PER_BLOCK - 1) / P_TOKENS_PER_BLOCK);
+    const size_t H = c.hidden, I = c.intermediate, EL = c.num_local_experts, rc = L.row_cap;
+    size_t o = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = o;
+        o = align_up(o + bytes);
+        return at;
+    };
+    L.topk_idx = take(slots * 4);
+    L.topk_w = take(slots * 4);
+    L.block_hist = take(static_cast<size_t>(L.max_blocks) * EL * 4);
+    L.expert_count = take(EL * 4);
+    L.expert_offset = take((EL + 1) * 4);
+    L.padded_offset = take((EL + 1) * 4);
+    L.tile_expert = take(static_cast<size_t>(L.max_m_tiles) * 4);
+    L.tile_rows = take(static_cast<size_t>(L.max_m_tiles) * 4);
+    L.num_m_tiles = take(4);
+    L.slot_to_row = take(slots * 4);
+    L.row_to_slot = take(slots * 4);
+    L.row_token = take(rc * 4);
+    L.status = take(4);
+    L.a1 = take(rc * H);
+    L.a1_scale_t = take(rc * (H / 128) * 4);
+    L.a2 = take(rc * I);
+    L.a2_scale_t = take(rc * (I / 128) * 4);
+    L.y = take(rc * H * 2);
+    L.stage_hidden = take(Tm * H);
+    L.stage_scale = take(Tm * (H / 128) * 4);
+    L.stage_logits = take(Tm * 256 * 4);
+    L.stage_out = take(Tm * H * 2);
+    L.total = o;
+    return L;
+}
+
+}  // namespace
+
+struct moe_fp8_handle_s {
+    moe_fp8_config cfg;
+    WsLayout L;
+    int sm_count;
+    int last_cuda_error;
+    int last_launches;
+    int last_T;
+    uint8_t* ws;
+    size_t ws_bytes;
+    EncodeTiledFn encode;
+    CUtensorMap tm_a1, tm_a2, tm_w13, tm_w2;
+    const void* w13_cached;
+    const void* w2_cached;
+};
+
+namespace {
+
+int cuda_fail(moe_fp8_handle_t h, cudaError_t e) {
+    if (h) h->last_cuda_error = static_cast<int>(e);
+    return MOE_FP8_ERR_CUDA;
+}
+
+// 2-D uint8 tensor [rows, cols] (cols contiguous), box 128 bytes x 128 rows, 128-byte swizzle.
+bool encode_2d(moe_fp8_handle_t h, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols) {
+    cuuint64_t gdim[2] = {cols, rows};
+    cuuint64_t gstride[1] = {cols};
+    cuuint32_t box[2] = {128, 128};
+    cuuint32_t estride[2] = {1, 1};
+    CUresult r = h->encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), gdim, gstride, box, estride,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+template <typename T>
+T* at(moe_fp8_handle_t h, size_t off) {
+    return reinterpret_cast<T*>(h->ws + off);
+}
+
+PermuteMeta meta_of(moe_fp8_handle_t h) {
+    PermuteMeta m;
+    m.block_hist = at<int>(h, h->L.block_hist);
+    m.expert_count = at<int>(h, h->L.expert_count);
+    m.expert_offset = at<int>(h, h->L.expert_offset);
+    m.padded_offset = at<int>(h, h->L.padded_offset);
+    m.tile_expert = at<int>(h, h->L.tile_expert);
+    m.tile_rows = at<int>(h, h->L.tile_rows);
+    m.num_m_tiles = at<int>(h, h->L.num_m_tiles);
+    m.slot_to_row = at<int>(h, h->L.slot_to_row);
+    m.row_to_slot = at<int>(h, h->L.row_to_slot);
+    m.row_token = at<int>(h, h->L.row_token);
+    return m;
+}
+
+bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+// Debug: canonical row r -> padded row, then copy that row's intermediate results.
+__global__ void export_rows_kernel(int E_loc, int I, int H, int row_cap, const int* __restrict__ expert_offset,
+                                   const int* __restrict__ padded_offset, const uint8_t* __restrict__ a2,
+                                   const float* __restrict__ a2_scale_t, const __nv_bfloat16* __restrict__ y,
+                                   uint8_t* __restrict__ a2_out, float* __restrict__ a2_scale_out,
+                                   __nv_bfloat16* __restrict__ y_out) {
+    const int S = expert_offset[E_loc];
+    for (int r = blockIdx.x; r < S; r += gridDim.x) {
+        int e = 0;
+        while (e + 1 < E_loc && expert_offset[e + 1] <= r) ++e;
+        const size_t p = static_cast<size_t>(padded_offset[e]) + (r - expert_offset[e]);
+        if (a2_out)
+            for (int i = threadIdx.x; i < I; i += blockDim.x) a2_out[static_cast<size_t>(r) * I + i] = a2[p * I + i];
+        if (a2_scale_out)
+            for (int i = threadIdx.x; i < I / 128; i += blockDim.x)
+                a2_scale_out[static_cast<size_t>(r) * (I / 128) + i] = a2_scale_t[static_cast<size_t>(i) * row_cap + p];
+        if (y_out)
+            for (int i = threadIdx.x; i < H; i += blockDim.x) y_out[static_cast<size_t>(r) * H + i] = y[p * H + i];
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* moe_fp8_strerror(int rc) {
+    switch (rc) {
+        case MOE_FP8_OK: return "ok";
+        case MOE_FP8_ERR_BAD_ARG: return "bad argument";
+        case MOE_FP8_ERR_UNSUPPORTED_DIMS: return "unsupported layer dimensions";
+        case MOE_FP8_ERR_NO_WORKSPACE: return "workspace missing or too small";
+        case MOE_FP8_ERR_CUDA: return "CUDA error";
+        case MOE_FP8_ERR_ARCH: return "device is not compute capability 10.x (no fallback path exists)";
+        default: return "unknown error";
+    }
+}
+
+int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
+    if (!cfg || !out) return MOE_FP8_ERR_BAD_ARG;
+    *out = nullptr;
+    if (cfg->max_tokens < 0 || cfg->hidden <= 0 || cfg->intermediate <= 0 || cfg->num_local_experts <= 0)
+        return MOE_FP8_ERR_BAD_ARG;
+    if (cfg->num_experts != R_EXPERTS || cfg->n_group != R_GROUPS || cfg->topk_group != R_TOPK_GROUP ||
+        cfg->top_k != R_TOPK || cfg->hidden % G_TILE_N != 0 || cfg->intermediate % 128 != 0 ||
+        cfg->num_local_experts > P_MAX_LOCAL || cfg->max_tokens > (1 << 20) ||
+        (cfg->hidden_scale_layout != 0 && cfg->hidden_scale_layout != 1))
+        return MOE_FP8_ERR_UNSUPPORTED_DIMS;
+
+    int dev = 0, major = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
+    if (major != 10) return MOE_FP8_ERR_ARCH;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
+
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) return MOE_FP8_ERR_CUDA;
+
+    e = cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
+    e = cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
+
+    moe_fp8_handle_s* h = new (std::nothrow) moe_fp8_handle_s();
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    memset(h, 0, sizeof(*h));
+    h->cfg = *cfg;
+    h->L = make_layout(*cfg);
+    h->sm_count = sms;
+    h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    *out = h;
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_destroy(moe_fp8_handle_t h) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    delete h;
+    return MOE_FP8_OK;
+}
+
+size_t moe_fp8_workspace_bytes(moe_fp8_handle_t h) { return h ? h->L.total : 0; }
+
+int moe_fp8_set_workspace(moe_fp8_handle_t h, void* ws, size_t bytes) {
+    if (!h || !ws || (reinterpret_cast<uintptr_t>(ws) % WS_ALIGN) != 0) return MOE_FP8_ERR_BAD_ARG;
+    if (bytes < h->L.total) return MOE_FP8_ERR_NO_WORKSPACE;
+    h->ws = static_cast<uint8_t*>(ws);
+    h->ws_bytes = bytes;
+    if (!encode_2d(h, &h->tm_a1, h->ws + h->L.a1, h->L.row_cap, h->cfg.hidden) ||
+        !encode_2d(h, &h->tm_a2, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate)) {
+        h->ws = nullptr;
+        return cuda_fail(h, cudaErrorInvalidValue);
+    }
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_last_cuda_error(moe_fp8_handle_t h) { return h ? h->last_cuda_error : 0; }
+int moe_fp8_last_launch_count(moe_fp8_handle_t h) { return h ? h->last_launches : 0; }
+
+int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const float* hidden_scale,
+                    const float* router_logits, const void* routing_bias, const void* w13, const float* w13_scale,
+                    const void* w2, const float* w2_scale, int local_expert_offset, float scaling_factor, void* out,
+                    void* stream_v) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    const moe_fp8_config& c = h->cfg;
+    if (T < 0 || T > c.max_tokens) return MOE_FP8_ERR_BAD_ARG;
+    if (local_expert_offset < 0 || local_expert_offset + c.num_local_experts > c.num_experts)
+        return MOE_FP8_ERR_BAD_ARG;
+    if (!routing_bias || !w13 || !w13_scale || !w2 || !w2_scale || misaligned(routing_bias) || misaligned(w13) ||
+        misaligned(w13_scale) || misaligned(w2) || misaligned(w2_scale))
+        return MOE_FP8_ERR_BAD_ARG;
+    if (T > 0 && (!hidden_fp8 || !hidden_scale || !router_logits || !out || misaligned(hidden_fp8) ||
+                  misaligned(hidden_scale) || misaligned(router_logits) || misaligned(out)))
+        return MOE_FP8_ERR_BAD_ARG;
+    if (!h->ws) return MOE_FP8_ERR_NO_WORKSPACE;
+    h->last_launches = 0;
+    h->last_T = T;
+    if (T == 0) return MOE_FP8_OK;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int H = c.hidden, I = c.intermediate, EL = c.num_local_experts;
+    if (w13 != h->w13_cached || w2 != h->w2_cached) {
+        if (!encode_2d(h, &h->tm_w13, w13, static_cast<uint64_t>(EL) * 2 * I, H) ||
+            !encode_2d(h, &h->tm_w2, w2, static_cast<uint64_t>(EL) * H, I))
+            return cuda_fail(h, cudaErrorInvalidValue);
+        h->w13_cached = w13;
+        h->w2_cached = w2;
+    }
+
+    PermuteMeta m = meta_of(h);
+    int* topk_idx = at<int>(h, h->L.topk_idx);
+    float* topk_w = at<float>(h, h->L.topk_w);
+    int* status = at<int>(h, h->L.status);
+    uint8_t* a1 = at<uint8_t>(h, h->L.a1);
+    float* a1_scale_t = at<float>(h, h->L.a1_scale_t);
+    uint8_t* a2 = at<uint8_t>(h, h->L.a2);
+    float* a2_scale_t = at<float>(h, h->L.a2_scale_t);
+    __nv_bfloat16* y = at<__nv_bfloat16>(h, h->L.y);
+    const int row_cap = h->L.row_cap;
+    const int nblk = (T + P_TOKENS_PER_BLOCK - 1) / P_TOKENS_PER_BLOCK;
+    int launches = 0;
+
+    cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+
+    {  // stage 1: routing
+        const int grid = min((T + 7) / 8, h->sm_count * 8);
+        route_topk_kernel<<<grid, 256, 0, stream>>>(T, router_logits, static_cast<const __nv_bfloat16*>(routing_bias),
+                                                    scaling_factor, topk_idx, topk_w);
+        ++launches;
+    }
+    {  // stage 2: histogram, scan, placement, gather
+        count_kernel<<<nblk, P_TOKENS_PER_BLOCK, 0, stream>>>(T, EL, local_expert_offset, topk_idx, m.block_hist);
+        scan_kernel<<<1, P_MAX_LOCAL, 0, stream>>>(nblk, EL, m);
+        place_kernel<<<nblk, P_TOKENS_PER_BLOCK, 0, stream>>>(T, EL, local_expert_offset, row_cap, topk_idx, m,
+                                                              status);
+        const long long row_bound = static_cast<long long>(T) * 8 + static_cast<long long>(EL) * (TILE_M - 1);
+        const int grid = static_cast<int>(std::min<long long>((row_bound + 7) / 8, h->sm_count * 8LL));
+        gather_rows_kernel<<<grid, 256, 0, stream>>>(H, row_cap, c.hidden_scale_layout, T,
+                                                     static_cast<const uint8_t*>(hidden_fp8), hidden_scale, m, a1,
+                                                     a1_scale_t);
+        launches += 4;
+    }
+    {  // stage 3a: GEMM1 + SwiGLU + re-quantisation
+        GemmArgs g;
+        memset(&g, 0, sizeof(g));
+        g.num_kb = H / 128;
+        g.n_tiles = I / 128;
+        g.w_rows_per_expert = 2 * I;
+        g.row_cap = row_cap;
+        g.out_cols = I;
+        g.gate_row0 = c.gate_first ? 0 : I;
+        g.up_row0 = c.gate_first ? I : 0;
+        g.num_m_tiles = m.num_m_tiles;
+        g.tile_expert = m.tile_expert;
+        g.tile_rows = m.tile_rows;
+        g.a_scale_t = a1_scale_t;
+        g.w_scale = w13_scale;
+        g.out_fp8 = a2;
+        g.out_scale_t = a2_scale_t;
+        g.status = status;
+        grouped_gemm_kernel<1><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a1, h->tm_w13, g);
+        ++launches;
+    }
+    {  // stage 3b: GEMM2
+        GemmArgs g;
+        memset(&g, 0, sizeof(g));
+        g.num_kb = I / 128;
+        g.n_tiles = H / G_TILE_N;
+        g.w_rows_per_expert = H;
+        g.row_cap = row_cap;
+        g.out_cols = H;
+        g.num_m_tiles = m.num_m_tiles;
+        g.tile_expert = m.tile_expert;
+        g.tile_rows = m.tile_rows;
+        g.a_scale_t = a2_scale_t;
+        g.w_scale = w2_scale;
+        g.out_bf16 = y;
+        g.status = status;
+        grouped_gemm_kernel<2><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a2, h->tm_w2, g);
+        ++launches;
+    }
+    {  // stage 4: weighted combine back to token order
+        const int grid = min(T, h->sm_count * 16);
+        combine_kernel<<<grid, 256, 0, stream>>>(T, H, m.slot_to_row, topk_w, y, static_cast<__nv_bfloat16*>(out));
+        ++launches;
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->last_launches = launches;
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_forward_host(moe_fp8_handle_t h, int T, const void* host_hidden_fp8, const float* host_hidden_scale,
+                         const float* host_router_logits, const void* routing_bias, const void* w13,
+                         const float* w13_scale, const void* w2, const float* w2_scale, int local_expert_offset,
+                         float scaling_factor, void* host_out, void* stream_v) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    if (T < 0 || T > h->cfg.max_tokens) return MOE_FP8_ERR_BAD_ARG;
+    if (T > 0 && (!host_hidden_fp8 || !host_hidden_scale || !host_router_logits || !host_out))
+        return MOE_FP8_ERR_BAD_ARG;
+    if (!h->ws) return MOE_FP8_ERR_NO_WORKSPACE;
+    if (T == 0) return moe_fp8_forward(h, 0, nullptr, nullptr, nullptr, routing_bias, w13, w13_scale, w2, w2_scale,
+                                       local_expert_offset, scaling_factor, nullptr, stream_v);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t H = h->cfg.hidden, Tz = T;
+    uint8_t* d_hidden = at<uint8_t>(h, h->L.stage_hidden);
+    float* d_scale = at<float>(h, h->L.stage_scale);
+    float* d_logits = at<float>(h, h->L.stage_logits);
+    void* d_out = at<uint8_t>(h, h->L.stage_out);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(d_hidden, host_hidden_fp8, Tz * H, cudaMemcpyHostToDevice, stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(d_scale, host_hidden_scale, Tz * (H / 128) * 4, cudaMemcpyHostToDevice, stream)) !=
+            cudaSuccess ||
+        (e = cudaMemcpyAsync(d_logits, host_router_logits, Tz * 256 * 4, cudaMemcpyHostToDevice, stream)) !=
+            cudaSuccess)
+        return cuda_fail(h, e);
+    int rc = moe_fp8_forward(h, T, d_hidden, d_scale, d_logits, routing_bias, w13, w13_scale, w2, w2_scale,
+                             local_expert_offset, scaling_factor, d_out, stream_v);
+    if (rc != MOE_FP8_OK) return rc;
+    if ((e = cudaMemcpyAsync(host_out, d_out, Tz * H * 2, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return cuda_fail(h, e);
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(h, e);
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w, int* expert_count,
+                         int* expert_offset, int* row_to_slot, void* a2_fp8, float* a2_scale, void* y_rows,
+                         int* status_word, void* stream_v) {
+    if (!h || T < 0 || T > h->cfg.max_tokens) return MOE_FP8_ERR_BAD_ARG;
+    if (!h->ws) return MOE_FP8_ERR_NO_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t slots = static_cast<size_t>(T) * 8, EL = h->cfg.num_local_experts;
+    cudaError_t e = cudaSuccess;
+    auto copy = [&](void* dst, size_t off, size_t bytes) {
+        if (dst && bytes && e == cudaSuccess)
+            e = cudaMemcpyAsync(dst, h->ws + off, bytes, cudaMemcpyDeviceToDevice, stream);
+    };
+    copy(status_word, h->L.status, 4);
+    if (T > 0 && h->last_T == T) {
+        copy(topk_idx, h->L.topk_idx, slots * 4);
+        copy(topk_w, h->L.topk_w, slots * 4);
+        copy(expert_count, h->L.expert_count, EL * 4);
+        copy(expert_offset, h->L.expert_offset, (EL + 1) * 4);
+        copy(row_to_slot, h->L.row_to_slot, slots * 4);
+        if (e == cudaSuccess && (a2_fp8 || a2_scale || y_rows)) {
+            export_rows_kernel<<<1024, 256, 0, stream>>>(
+                static_cast<int>(EL), h->cfg.intermediate, h->cfg.hidden, h->L.row_cap,
+                at<int>(h, h->L.expert_offset), at<int>(h, h->L.padded_offset), at<uint8_t>(h, h->L.a2),
+                at<float>(h, h->L.a2_scale_t), at<__nv_bfloat16>(h, h->L.y), static_cast<uint8_t*>(a2_fp8), a2_scale,
+                static_cast<__nv_bfloat16*>(y_rows));
+            e = cudaGetLastError();
+        }
+    } else if (T > 0) {
+        return MOE_FP8_ERR_BAD_ARG;
+    }
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return MOE_FP8_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,168 @@
+// Stage 2 of the Fused MoE description: per-expert histogram, exclusive scan,
+// stable placement of the local (token, expert) slots into expert-contiguous
+// rows (experts ascending, tokens ascending inside an expert), and the gather
+// of FP8 activation rows and their 128-wide scales into that order.  All
+// metadata stays on the device; nothing here synchronises with the host.
+//
+// Row numbering: "canonical" rows are dense (expert e starts at offset[e]);
+// "padded" rows start every expert on a multiple of the GEMM tile height so a
+// tile never straddles two experts.
+#pragma once
+#include <stdint.h>
+
+namespace moe {
+
+constexpr int P_TOKENS_PER_BLOCK = 256;  // tokens handled by one block of the count/place kernels
+constexpr int P_MAX_LOCAL = 256;         // most local experts supported
+constexpr int TILE_M = 128;              // GEMM tile height (rows)
+
+struct PermuteMeta {
+    int* block_hist;     // [nblk, E_loc] per-block counts, turned into per-block bases by the scan
+    int* expert_count;   // [E_loc]
+    int* expert_offset;  // [E_loc+1] canonical (unpadded) exclusive scan
+    int* padded_offset;  // [E_loc+1] exclusive scan of counts rounded up to TILE_M
+    int* tile_expert;    // [max_m_tiles] local expert of each row tile
+    int* tile_rows;      // [max_m_tiles] valid rows in each row tile (1..TILE_M)
+    int* num_m_tiles;    // [1]
+    int* slot_to_row;    // [T*8] padded row of each slot, -1 when the slot's expert is not local
+    int* row_to_slot;    // [T*8] canonical row -> slot id (first S entries valid)
+    int* row_token;      // [row_cap] padded row -> token (valid rows only)
+};
+
+// Bit t of mask[e] says: token t of this block routes to local expert e.  The
+// popcount below a token's bit is its stable rank inside the block.
+__device__ __forceinline__ void build_block_masks(uint32_t (*mask)[P_TOKENS_PER_BLOCK / 32], int T, int E_loc,
+                                                  int off, const int* __restrict__ topk_idx) {
+    for (int i = threadIdx.x; i < E_loc * (P_TOKENS_PER_BLOCK / 32); i += blockDim.x)
+        (&mask[0][0])[i] = 0u;
+    __syncthreads();
+    const int t = blockIdx.x * P_TOKENS_PER_BLOCK + threadIdx.x;
+    if (t < T) {
+        const int4 a = reinterpret_cast<const int4*>(topk_idx)[2 * t];
+        const int4 b = reinterpret_cast<const int4*>(topk_idx)[2 * t + 1];
+        const int ids[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int e = ids[j] - off;
+            if (e >= 0 && e < E_loc) atomicOr(&mask[e][threadIdx.x >> 5], 1u << (threadIdx.x & 31));
+        }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) count_kernel(int T, int E_loc, int off,
+                                                                   const int* __restrict__ topk_idx,
+                                                                   int* __restrict__ block_hist) {
+    __shared__ uint32_t mask[P_MAX_LOCAL][P_TOKENS_PER_BLOCK / 32];
+    build_block_masks(mask, T, E_loc, off, topk_idx);
+    for (int e = threadIdx.x; e < E_loc; e += blockDim.x) {
+        int c = 0;
+#pragma unroll
+        for (int w = 0; w < P_TOKENS_PER_BLOCK / 32; ++w) c += __popc(mask[e][w]);
+        block_hist[blockIdx.x * E_loc + e] = c;
+    }
+}
+
+// One block.  Thread e owns local expert e.
+__global__ void __launch_bounds__(P_MAX_LOCAL) scan_kernel(int nblk, int E_loc, PermuteMeta m) {
+    __shared__ int s_cnt[P_MAX_LOCAL + 1];
+    __shared__ int s_pad[P_MAX_LOCAL + 1];
+    const int e = threadIdx.x;
+    int total = 0;
+    if (e < E_loc) {
+        for (int b = 0; b < nblk; ++b) {
+            const int c = m.block_hist[b * E_loc + e];
+            m.block_hist[b * E_loc + e] = total;  // base of block b inside expert e
+            total += c;
+        }
+    }
+    s_cnt[e] = (e < E_loc) ? total : 0;
+    s_pad[e] = (e < E_loc) ? (total + TILE_M - 1) / TILE_M * TILE_M : 0;
+    __syncthreads();
+    if (threadIdx.x == 0) {  // 256 entries: a serial scan is a few hundred cycles
+        int a = 0, p = 0;
+        for (int i = 0; i < E_loc; ++i) {
+            const int c = s_cnt[i], q = s_pad[i];
+            s_cnt[i] = a;
+            s_pad[i] = p;
+            a += c;
+            p += q;
+        }
+        s_cnt[E_loc] = a;
+        s_pad[E_loc] = p;
+        *m.num_m_tiles = p / TILE_M;
+    }
+    __syncthreads();
+    if (e < E_loc) {
+        m.expert_count[e] = total;
+        m.expert_offset[e] = s_cnt[e];
+        m.padded_offset[e] = s_pad[e];
+        const int t0 = s_pad[e] / TILE_M;
+        for (int i = 0; i * TILE_M < total; ++i) {
+            m.tile_expert[t0 + i] = e;
+            m.tile_rows[t0 + i] = min(TILE_M, total - i * TILE_M);
+        }
+    }
+    if (e == 0) {
+        m.expert_offset[E_loc] = s_cnt[E_loc];
+        m.padded_offset[E_loc] = s_pad[E_loc];
+    }
+}
+
+__global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) place_kernel(int T, int E_loc, int off, int row_cap,
+                                                                   const int* __restrict__ topk_idx, PermuteMeta m,
+                                                                   int* __restrict__ status) {
+    __shared__ uint32_t mask[P_MAX_LOCAL][P_TOKENS_PER_BLOCK / 32];
+    build_block_masks(mask, T, E_loc, off, topk_idx);
+    const int t = blockIdx.x * P_TOKENS_PER_BLOCK + threadIdx.x;
+    if (t >= T) return;
+    const int word = threadIdx.x >> 5, bit = threadIdx.x & 31;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int e = topk_idx[t * 8 + j] - off;
+        int prow = -1;
+        if (e >= 0 && e < E_loc) {
+            int rank = __popc(mask[e][word] & ((1u << bit) - 1u));
+            for (int w = 0; w < word; ++w) rank += __popc(mask[e][w]);
+            const int within = m.block_hist[blockIdx.x * E_loc + e] + rank;
+            prow = m.padded_offset[e] + within;
+            if (prow < 0 || prow >= row_cap) {
+                atomicExch(status, DEV_BAD_ROW);
+                prow = -1;
+            } else {
+                m.row_to_slot[m.expert_offset[e] + within] = t * 8 + j;
+                m.row_token[prow] = t;
+            }
+        }
+        m.slot_to_row[t * 8 + j] = prow;
+    }
+}
+
+// One warp per padded row: copy the token's FP8 row (K bytes) and write its
+// K/128 scales transposed ([K/128, row_cap]) so the GEMM epilogue reads them
+// coalesced across the rows of a tile.  Rows past an expert's count are padding
+// and are left untouched (their results are never stored).
+__global__ void __launch_bounds__(256) gather_rows_kernel(int H, int row_cap, int scale_layout, int T,
+                                                          const uint8_t* __restrict__ hidden,
+                                                          const float* __restrict__ hidden_scale, PermuteMeta m,
+                                                          uint8_t* __restrict__ a1, float* __restrict__ a1_scale_t) {
+    const int lane = threadIdx.x & 31;
+    const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int nwarps = gridDim.x * (blockDim.x >> 5);
+    const int rows = *m.num_m_tiles * TILE_M;
+    const int chunks = H / 16, nkb = H / 128;
+    for (int r = warp; r < rows; r += nwarps) {
+        if ((r % TILE_M) >= m.tile_rows[r / TILE_M]) continue;
+        const int t = m.row_token[r];
+        const uint4* src = reinterpret_cast<const uint4*>(hidden + static_cast<size_t>(t) * H);
+        uint4* dst = reinterpret_cast<uint4*>(a1 + static_cast<size_t>(r) * H);
+        for (int c = lane; c < chunks; c += 32) dst[c] = __ldg(src + c);
+        for (int kb = lane; kb < nkb; kb += 32) {
+            const float s = scale_layout ? hidden_scale[static_cast<size_t>(kb) * T + t]
+                                         : hidden_scale[static_cast<size_t>(t) * nkb + kb];
+            a1_scale_t[static_cast<size_t>(kb) * row_cap + r] = s;
+        }
+    }
+}
+
+}  // namespace moe

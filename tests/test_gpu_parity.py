@@ -1,0 +1,150 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle
+on the same seeded inputs.  Routing indices and the permutation are compared
+bit for bit, the bf16 output with the tolerance of the workload definition."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_14560_b200 import MoeFp8, MoeFp8Error
+from paper_2608_14560_b200 import synthetic as syn
+
+from parity import check_output, make_engine, run_and_compare
+
+pytestmark = pytest.mark.gpu
+
+SMALL = syn.LayerDims(hidden=512, intermediate=256, num_local_experts=32)
+
+
+def _wl(tokens, dims=SMALL, seed=0, **kw):
+    return syn.Workload(f"t{tokens}", tokens, dims, seed, **kw)
+
+
+# ---- small layer, every token compared ------------------------------------
+@pytest.mark.parametrize("tokens", [1, 7, 130, 1000])
+def test_small_layer_all_tokens(cuda_device, tokens):
+    st = run_and_compare(_wl(tokens, seed=tokens), cuda_device)
+    assert st["frac"] >= 0.995
+
+
+def test_small_layer_skewed_many_tiles_per_expert(cuda_device):
+    # hot experts receive every token: several 128-row tiles per expert plus a ragged tail
+    st = run_and_compare(_wl(1111, seed=9, skew=True), cuda_device)
+    assert st["S"] > 4 * 1111
+
+
+def test_all_experts_local(cuda_device):
+    dims = dataclasses.replace(SMALL, num_local_experts=256)
+    st = run_and_compare(_wl(333, dims, seed=5), cuda_device)
+    assert st["S"] == 333 * 8
+
+
+@pytest.mark.parametrize("off,eloc", [(32, 32), (224, 32), (5, 3), (0, 1)])
+def test_local_expert_offsets(cuda_device, off, eloc):
+    dims = dataclasses.replace(SMALL, num_local_experts=eloc)
+    run_and_compare(_wl(200, dims, seed=off + eloc, local_expert_offset=off), cuda_device)
+
+
+def test_scale_layout_and_gate_order_flags(cuda_device):
+    wl = _wl(97, seed=3)
+    inp = syn.make_inputs(wl, cuda_device)
+    inp_t = dict(inp, hidden_scale=inp["hidden_scale"].t().contiguous())
+    run_and_compare(wl, cuda_device, inp=inp_t, hidden_scale_layout=1)
+    I = wl.dims.intermediate
+    inp_s = dict(inp, w13=torch.cat([inp["w13"][:, I:], inp["w13"][:, :I]], 1).contiguous(),
+                 w13_scale=torch.cat([inp["w13_scale"][:, I // 128:], inp["w13_scale"][:, :I // 128]], 1).contiguous())
+    run_and_compare(wl, cuda_device, inp=inp_s, gate_first=False)
+
+
+# ---- degenerate cases -------------------------------------------------------
+def test_zero_tokens_and_argument_errors(cuda_device):
+    wl = _wl(0)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device, max_tokens=16)
+    out = eng.forward(inp)
+    assert out.shape == (0, 512) and eng.last_launch_count() == 0
+    big = syn.make_inputs(_wl(17), cuda_device)
+    with pytest.raises(MoeFp8Error) as ei:
+        eng.forward(big)  # T > max_tokens
+    assert ei.value.rc == -1
+    with pytest.raises(MoeFp8Error):
+        eng.forward(dict(syn.make_inputs(_wl(4), cuda_device), local_expert_offset=250))
+    with pytest.raises(MoeFp8Error):
+        MoeFp8(hidden=500, device=cuda_device)
+    eng.close()
+
+
+def test_no_token_routes_locally(cuda_device):
+    wl = _wl(64, seed=1)
+    inp = syn.make_inputs(wl, cuda_device)
+    inp["router_logits"][:, :32] = -20.0  # local experts (group 0) never win
+    st = run_and_compare(wl, cuda_device, inp=inp)
+    assert st["S"] == 0
+
+
+def test_every_token_on_the_same_experts(cuda_device):
+    wl = _wl(300, seed=2)
+    inp = syn.make_inputs(wl, cuda_device)
+    inp["router_logits"][:] = -8.0
+    inp["router_logits"][:, [1, 2, 3, 4, 40, 41, 80, 120]] = 6.0
+    st = run_and_compare(wl, cuda_device, inp=inp)
+    assert st["S"] == 4 * 300 and st["active"] == 4
+
+
+def test_exact_score_ties_break_to_smaller_index(cuda_device):
+    wl = _wl(50, seed=4)
+    inp = syn.make_inputs(wl, cuda_device)
+    inp["router_logits"][:] = 0.25
+    inp["routing_bias"][:] = 0
+    run_and_compare(wl, cuda_device, inp=inp)
+    inp["router_logits"][:, 128:] = 0.5  # ties inside and across groups 4..7
+    run_and_compare(wl, cuda_device, inp=inp)
+
+
+def test_run_to_run_determinism_and_workspace_reuse(cuda_device):
+    wl = _wl(500, seed=6)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device, max_tokens=600)
+    a = eng.forward(inp).clone()
+    other = syn.make_inputs(_wl(77, seed=8), cuda_device)
+    eng.forward(other)  # different T in between: stale scratch must not leak
+    b = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    run_and_compare(_wl(77, seed=8), cuda_device, inp=other, eng=eng)
+    eng.close()
+
+
+def test_host_entry_point_matches_device_entry_point(cuda_device):
+    wl = _wl(260, seed=12)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device)
+    ref = eng.forward(inp).cpu()
+    host_act = {k: inp[k].cpu().pin_memory() for k in ("hidden_fp8", "hidden_scale", "router_logits")}
+    host_out = torch.empty(wl.tokens, 512, dtype=torch.bfloat16).pin_memory()
+    eng.forward_host(host_act, inp, host_out)
+    assert torch.equal(ref.view(torch.int16), host_out.view(torch.int16))
+    eng.close()
+
+
+# ---- the five benchmark workloads at full size -----------------------------
+def _sample(T, n, seed):
+    if T <= n:
+        return None
+    return np.sort(np.random.default_rng(seed).choice(T, n, replace=False)).astype(np.int32)
+
+
+@pytest.mark.parametrize("cfg,n_sample", [(0, 8), (1, 64), (2, 256), (3, 40)])
+def test_benchmark_workloads_32_local_experts(cuda_device, cfg, n_sample):
+    wl = syn.CONFIGS[cfg]
+    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(wl.tokens, n_sample, cfg))
+    print(wl.name, st)
+
+
+def test_benchmark_workload_all_256_experts_local(cuda_device):
+    wl = syn.CONFIGS[4]
+    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(wl.tokens, 24, 4))
+    assert st["S"] == wl.tokens * 8
+    print(wl.name, st)
