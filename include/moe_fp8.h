@@ -125,6 +125,22 @@ int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w
                          int* expert_offset, int* row_to_slot, void* a2_fp8, float* a2_scale, void* y_rows,
                          int* status_word, void* stream);
 
+/*
+ * Measurement hook (the paper profiles each kernel of one MoE iteration, Appendix
+ * "NCU Profile of the Slowest FuseMoE Workload"): when enabled, moe_fp8_forward
+ * records a CUDA event on `stream` before and after each of its kernel launches.
+ * Enabling creates the events (not for use inside the hot path); disabling
+ * destroys them.  Off by default.
+ */
+int moe_fp8_set_stage_timing(moe_fp8_handle_t h, int enable);
+/* Number of stages and the name of stage i ("route_topk", ..., "combine"). */
+int moe_fp8_num_stages(void);
+const char* moe_fp8_stage_name(int i);
+/* Waits for the events of the last forward and writes the device time of each
+ * stage in milliseconds to host_ms[0..n) (host pointer); returns the number of
+ * stages written. */
+int moe_fp8_get_stage_times(moe_fp8_handle_t h, float* host_ms, int n);
+
 /* CUDA error code (cudaError_t as int) of the last MOE_FP8_ERR_CUDA on this handle. */
 int moe_fp8_last_cuda_error(moe_fp8_handle_t h);
 /* Kernel launches enqueued by the last moe_fp8_forward on this handle. */

@@ -16,7 +16,8 @@ ERR_BAD_ARG, ERR_UNSUPPORTED_DIMS, ERR_NO_WORKSPACE, ERR_CUDA, ERR_ARCH = -1, -2
 EXPORTS = (
     "moe_fp8_create", "moe_fp8_destroy", "moe_fp8_workspace_bytes", "moe_fp8_set_workspace", "moe_fp8_forward",
     "moe_fp8_forward_host", "moe_fp8_debug_export", "moe_fp8_last_cuda_error", "moe_fp8_last_launch_count",
-    "moe_fp8_strerror",
+    "moe_fp8_strerror", "moe_fp8_set_stage_timing", "moe_fp8_num_stages", "moe_fp8_stage_name",
+    "moe_fp8_get_stage_times",
 )
 
 
@@ -63,6 +64,14 @@ def load_library() -> C.CDLL:
         lib.moe_fp8_last_cuda_error.restype = C.c_int
         lib.moe_fp8_last_launch_count.argtypes = [vp]
         lib.moe_fp8_last_launch_count.restype = C.c_int
+        lib.moe_fp8_set_stage_timing.argtypes = [vp, C.c_int]
+        lib.moe_fp8_set_stage_timing.restype = C.c_int
+        lib.moe_fp8_num_stages.argtypes = []
+        lib.moe_fp8_num_stages.restype = C.c_int
+        lib.moe_fp8_stage_name.argtypes = [C.c_int]
+        lib.moe_fp8_stage_name.restype = C.c_char_p
+        lib.moe_fp8_get_stage_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int]
+        lib.moe_fp8_get_stage_times.restype = C.c_int
         lib.moe_fp8_strerror.argtypes = [C.c_int]
         lib.moe_fp8_strerror.restype = C.c_char_p
         _lib = lib
@@ -137,6 +146,21 @@ class MoeFp8:
             int(weights["local_expert_offset"]), float(weights["scaling_factor"]), _ptr(host_out),
             self._stream(stream)))
         return host_out
+
+    def set_stage_timing(self, enable: bool):
+        self._check(self.lib.moe_fp8_set_stage_timing(self.handle, int(enable)))
+
+    def stage_names(self):
+        return [self.lib.moe_fp8_stage_name(i).decode() for i in range(self.lib.moe_fp8_num_stages())]
+
+    def get_stage_times(self) -> dict:
+        """Device milliseconds per kernel of the last forward (stage timing must be on)."""
+        n = self.lib.moe_fp8_num_stages()
+        buf = (C.c_float * n)()
+        k = self.lib.moe_fp8_get_stage_times(self.handle, buf, n)
+        if k < 0:
+            self._check(k)
+        return dict(zip(self.stage_names(), list(buf)[:k]))
 
     def last_launch_count(self) -> int:
         return int(self.lib.moe_fp8_last_launch_count(self.handle))

@@ -90,6 +90,9 @@ struct moe_fp8_handle_s {
     CUtensorMap tm_a1, tm_a2, tm_w13, tm_w2;
     const void* w13_cached;
     const void* w2_cached;
+    bool stage_timing;
+    bool stage_times_valid;
+    cudaEvent_t ev[9];
 };
 
 namespace {
@@ -130,6 +133,10 @@ PermuteMeta meta_of(moe_fp8_handle_t h) {
     m.row_token = at<int>(h, h->L.row_token);
     return m;
 }
+
+constexpr int NUM_STAGES = 8;
+const char* const STAGE_NAMES[NUM_STAGES] = {"route_topk", "count", "scan", "place", "gather_rows",
+                                             "gemm1_swiglu_quant", "gemm2", "combine"};
 
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -213,6 +220,7 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
 
 int moe_fp8_destroy(moe_fp8_handle_t h) {
     if (!h) return MOE_FP8_ERR_BAD_ARG;
+    moe_fp8_set_stage_timing(h, 0);
     delete h;
     return MOE_FP8_OK;
 }
@@ -280,24 +288,35 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
 
     cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), stream);
     if (e != cudaSuccess) return cuda_fail(h, e);
+    int ev_i = 0;
+    auto mark = [&]() {
+        if (h->stage_timing) cudaEventRecord(h->ev[ev_i++], stream);
+    };
+    h->stage_times_valid = false;
+    mark();
 
     {  // stage 1: routing
         const int grid = min((T + 7) / 8, h->sm_count * 8);
         route_topk_kernel<<<grid, 256, 0, stream>>>(T, router_logits, static_cast<const __nv_bfloat16*>(routing_bias),
                                                     scaling_factor, topk_idx, topk_w);
         ++launches;
+        mark();
     }
     {  // stage 2: histogram, scan, placement, gather
         count_kernel<<<nblk, P_TOKENS_PER_BLOCK, 0, stream>>>(T, EL, local_expert_offset, topk_idx, m.block_hist);
+        mark();
         scan_kernel<<<1, P_MAX_LOCAL, 0, stream>>>(nblk, EL, m);
+        mark();
         place_kernel<<<nblk, P_TOKENS_PER_BLOCK, 0, stream>>>(T, EL, local_expert_offset, row_cap, topk_idx, m,
                                                               status);
+        mark();
         const long long row_bound = static_cast<long long>(T) * 8 + static_cast<long long>(EL) * (TILE_M - 1);
         const int grid = static_cast<int>(std::min<long long>((row_bound + 7) / 8, h->sm_count * 8LL));
         gather_rows_kernel<<<grid, 256, 0, stream>>>(H, row_cap, c.hidden_scale_layout, T,
                                                      static_cast<const uint8_t*>(hidden_fp8), hidden_scale, m, a1,
                                                      a1_scale_t);
         launches += 4;
+        mark();
     }
     {  // stage 3a: GEMM1 + SwiGLU + re-quantisation
         GemmArgs g;
@@ -319,6 +338,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         g.status = status;
         grouped_gemm_kernel<1><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a1, h->tm_w13, g);
         ++launches;
+        mark();
     }
     {  // stage 3b: GEMM2
         GemmArgs g;
@@ -337,16 +357,56 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         g.status = status;
         grouped_gemm_kernel<2><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a2, h->tm_w2, g);
         ++launches;
+        mark();
     }
     {  // stage 4: weighted combine back to token order
         const int grid = min(T, h->sm_count * 16);
         combine_kernel<<<grid, 256, 0, stream>>>(T, H, m.slot_to_row, topk_w, y, static_cast<__nv_bfloat16*>(out));
         ++launches;
+        mark();
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches = launches;
+    h->stage_times_valid = h->stage_timing;
     return MOE_FP8_OK;
+}
+
+int moe_fp8_set_stage_timing(moe_fp8_handle_t h, int enable) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    if ((enable != 0) == h->stage_timing) return MOE_FP8_OK;
+    h->stage_times_valid = false;
+    if (enable) {
+        for (int i = 0; i <= NUM_STAGES; ++i) {
+            cudaError_t e = cudaEventCreate(&h->ev[i]);
+            if (e != cudaSuccess) {
+                for (int j = 0; j < i; ++j) cudaEventDestroy(h->ev[j]);
+                return cuda_fail(h, e);
+            }
+        }
+        h->stage_timing = true;
+    } else {
+        for (int i = 0; i <= NUM_STAGES; ++i) cudaEventDestroy(h->ev[i]);
+        h->stage_timing = false;
+    }
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_num_stages(void) { return NUM_STAGES; }
+
+const char* moe_fp8_stage_name(int i) { return (i >= 0 && i < NUM_STAGES) ? STAGE_NAMES[i] : ""; }
+
+int moe_fp8_get_stage_times(moe_fp8_handle_t h, float* host_ms, int n) {
+    if (!h || !host_ms || n < 0) return MOE_FP8_ERR_BAD_ARG;
+    if (!h->stage_timing || !h->stage_times_valid) return MOE_FP8_ERR_BAD_ARG;
+    cudaError_t e = cudaEventSynchronize(h->ev[NUM_STAGES]);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    const int k = n < NUM_STAGES ? n : NUM_STAGES;
+    for (int i = 0; i < k; ++i) {
+        e = cudaEventElapsedTime(&host_ms[i], h->ev[i], h->ev[i + 1]);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    return k;
 }
 
 int moe_fp8_forward_host(moe_fp8_handle_t h, int T, const void* host_hidden_fp8, const float* host_hidden_scale,
