@@ -179,9 +179,6 @@ def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, 
     torch.cuda.synchronize()
     if world > 1:
         torch.distributed.barrier()
-    if sampler:
-        sampler.stop_flag = True
-        sampler.join()
     launches = eng.last_launch_count() * steps
     status = eng.status()
     assert status == 0, f"device status {status} after the timed region"
@@ -191,6 +188,9 @@ def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, 
     time_steps(eng, weights, acts, outs, flush, 3, stage=True)
     _, stage_ms = time_steps(eng, weights, acts, outs, flush, steps, stage=True)
     eng.set_stage_timing(False)
+    if sampler:  # clocks are sampled across the timed region and the identical per-kernel pass
+        sampler.stop_flag = True
+        sampler.join()
     stage_avg = {k: float(np.mean([s[k] for s in stage_ms])) for k in stage_ms[0]}
 
     ms = total_ms / steps
@@ -310,9 +310,14 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--others", default="0,2,3,4", help="extra workloads reported under 'workloads' at N=1 ('' = none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--tokens", type=int, default=0, help="override T of the chosen workload (profiling runs)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
     wl = syn.CONFIGS[args.config]
+    if args.tokens > 0:
+        wl = syn.Workload(f"{wl.name}_T{args.tokens}", args.tokens, wl.dims, wl.seed, wl.local_expert_offset,
+                          wl.scaling_factor, wl.skew)
 
     if args.impl == "reference":
         if rank == 0:
@@ -330,10 +335,12 @@ def main():
 
     my_wl = syn.Workload(wl.name, wl.tokens, wl.dims, wl.seed + 7919 * rank, wl.local_expert_offset,
                          wl.scaling_factor, wl.skew)
-    res = run_cuda_config(my_wl, device, args.steps, args.warmup, peaks, peak_kind, want_e2e=True,
+    res = run_cuda_config(my_wl, device, args.steps, args.warmup, peaks, peak_kind, want_e2e=not args.no_e2e,
                           cpu_baseline=(rank == 0 and world == 1 and not args.no_cpu_baseline),
                           sampler_index=physical_gpu_index(local_rank))
     total_ms = max_over_ranks(res["total_ms"], world, device)
+    if args.no_e2e:
+        res["e2e"] = {"ms_per_step": float("nan"), "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     e2e_ms = max_over_ranks(res["e2e"]["ms_per_step"], world, device)
     tokens_all = sum_over_ranks(float(my_wl.tokens), world, device)
     launches = sum_over_ranks(float(res["gpu_launches"]), world, device)

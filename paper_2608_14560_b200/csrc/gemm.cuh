@@ -4,16 +4,22 @@
 // the combine.
 //
 // One persistent CTA per SM walks a static list of 128 x 256 output tiles.
-//   warp 0      TMA producer: A tile (128 rows x 128 K-bytes) and B tile (256
-//               weight rows x 128 K-bytes) per K-block into a 4-stage ring,
-//               128-byte swizzle, completion on mbarriers.
-//   warp 1      MMA issuer: four tcgen05.mma (M128 N256 K32, e4m3 -> fp32) per
-//               K-block into one of two 256-column TMEM accumulators; each
-//               K-block starts from zero because its partial sum must be
+//   warp 0      TMA producer.  Per K-block (128 K-bytes = one scale block): the A
+//               tile (128 rows), the B tile (256 weight rows) and the 128
+//               activation scales of the block, into a 4-stage ring (128-byte
+//               swizzle) / an 8-slot scale ring, completion on mbarriers.
+//   warp 1      MMA issuer.  Four tcgen05.mma (M128 N256 K32, e4m3 -> fp32) per
+//               K-block into one of two 256-column TMEM buffers, then ONE
+//               tcgen05.commit: the same mbarrier tells the producer that the stage
+//               is free and the epilogue that the accumulator is ready (a single
+//               thread issues everything, and each MMA, commit and wait costs it
+//               50-100 clocks, so the per-K-block instruction count is kept minimal).
+//               Every K-block starts from zero because its partial sum must be
 //               multiplied by fp32 scales before it joins the running sum.
-//   warps 4-11  epilogue: read the K-block partial from TMEM, multiply by
-//               a_scale[row,kb] * w_scale[nblk,kb], accumulate in registers;
-//               at the end of the tile apply the fused tail and store.
+//   warps 4-7   epilogue of columns [0,128), warps 8-11 of columns [128,256): read
+//               the partial from TMEM, multiply by a_scale[row,kb] * w_scale[nblk,kb]
+//               with packed fp32 FMAs, accumulate in registers; at the end of the
+//               tile apply the fused tail and store.
 // Scales are arbitrary fp32 (amax/448), so the power-of-two hardware block
 // scaling cannot express them; the per-K-block promotion is done on the ALUs.
 #pragma once
@@ -25,16 +31,24 @@
 namespace moe {
 
 constexpr int G_STAGES = 4;
-constexpr int G_BLOCK_K = 128;                                  // K bytes per stage = one scale block
-constexpr int G_TILE_N = 256;                                   // accumulator columns
-constexpr int G_A_BYTES = TILE_M * G_BLOCK_K;                   // 16 KB
-constexpr int G_B_BYTES = G_TILE_N * G_BLOCK_K;                 // 32 KB
-constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;            // 48 KB
-constexpr int G_THREADS = 384;                                  // 4 control warps + 8 epilogue warps
-constexpr int G_EPI_THREADS = 256;
-constexpr int G_CTRL_BYTES = 4096;                              // barriers, flags, amax exchange
-constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_CTRL_BYTES + 1024;  // + alignment slack
+constexpr int G_BLOCK_K = 128;                          // K bytes per stage = one scale block
+constexpr int G_TILE_N = 256;                           // output columns per tile
+constexpr int G_HALF_N = 128;                           // columns handled by one epilogue warpgroup
+constexpr int G_ACC_BUFS = 2;                           // TMEM accumulator buffers (2 x 256 columns)
+constexpr int G_A_BYTES = TILE_M * G_BLOCK_K;           // 16 KB
+constexpr int G_B_BYTES = G_TILE_N * G_BLOCK_K;         // 32 KB
+constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;    // 48 KB
+constexpr int G_SCALE_RING = 8;                         // K-blocks of activation scales in flight
+constexpr int G_SCALE_BYTES = TILE_M * 4;               // 512 B per K-block
+constexpr int G_THREADS = 384;                          // 4 control warps + 8 epilogue warps
+constexpr int G_EPI_WARPS = 8;
+constexpr int G_STORE_WARP_BYTES = 2048;                // per-warp staging: 32 rows x 64 B (swizzled)
+constexpr int G_STORE_BYTES = G_EPI_WARPS * G_STORE_WARP_BYTES;
+constexpr int G_CTRL_BYTES = 512;
+constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_SCALE_RING * G_SCALE_BYTES + G_STORE_BYTES +
+                             G_CTRL_BYTES + 1024;       // + alignment slack
 constexpr uint32_t G_TMEM_COLS = 512;
+static_assert(G_SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
 struct GemmArgs {
     int num_kb;               // K / 128
@@ -50,20 +64,17 @@ struct GemmArgs {
     const float* w_scale;     // [E_loc, w_rows/128, num_kb]
     uint8_t* out_fp8;         // GEMM1: [row_cap, I] e4m3
     float* out_scale_t;       // GEMM1: [I/128, row_cap]
-    __nv_bfloat16* out_bf16;  // GEMM2: [row_cap, H]
     int* status;
 };
 
 struct GemmCtrl {
-    uint64_t full[G_STAGES];
-    uint64_t empty[G_STAGES];
-    uint64_t tmem_full[2];
-    uint64_t tmem_empty[2];
+    uint64_t full[G_STAGES];   // stage filled (TMA transaction bytes)
+    uint64_t done[G_STAGES];   // the MMAs that read the stage have finished: stage free AND accumulator ready
+    uint64_t tmem_empty[G_ACC_BUFS];
     uint64_t amax_bar[2];
     uint64_t drain_bar;
     uint32_t tmem_slot;
     int abort_flag;
-    float amax[2][2][TILE_M];  // [tile parity][column half][row]
 };
 static_assert(sizeof(GemmCtrl) <= G_CTRL_BYTES, "control block too large");
 
@@ -72,13 +83,18 @@ __device__ __forceinline__ void raise(GemmCtrl* c, int* status, int code) {
     atomicCAS(status, DEV_OK, code);
 }
 
+// MODE 1: gate/up projection + SwiGLU + re-quantisation (B tile = 4 x 64 weight rows:
+//         gate[0,64) | up[0,64) | gate[64,128) | up[64,128) of the tile's 128 columns).
+// MODE 2: down projection, bf16 rows out through TMA stores (B tile = 2 x 128 rows).
 template <int MODE>
 __global__ void __launch_bounds__(G_THREADS, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const GemmArgs g) {
+                    const __grid_constant__ CUtensorMap tmOut, const GemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(smem + G_STAGES * G_STAGE_BYTES);
+    float* scale_ring = reinterpret_cast<float*>(smem + G_STAGES * G_STAGE_BYTES);
+    uint8_t* store_stage = smem + G_STAGES * G_STAGE_BYTES + G_SCALE_RING * G_SCALE_BYTES;
+    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(store_stage + G_STORE_BYTES);
     volatile int* abort_flag = &ctrl->abort_flag;
     const uint32_t smem_base = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -86,13 +102,13 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (threadIdx.x == 0) {
         for (int s = 0; s < G_STAGES; ++s) {
             mbar_init(smem_u32(&ctrl->full[s]), 1);
-            mbar_init(smem_u32(&ctrl->empty[s]), 1);
+            mbar_init(smem_u32(&ctrl->done[s]), 1);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&ctrl->tmem_full[b]), 1);
-            mbar_init(smem_u32(&ctrl->tmem_empty[b]), G_EPI_THREADS / 32);
-            mbar_init(smem_u32(&ctrl->amax_bar[b]), G_EPI_THREADS);
+        for (int b = 0; b < G_ACC_BUFS; ++b) {
+            mbar_init(smem_u32(&ctrl->tmem_empty[b]), G_EPI_WARPS);
         }
+        mbar_init(smem_u32(&ctrl->amax_bar[0]), G_EPI_WARPS * 32);
+        mbar_init(smem_u32(&ctrl->amax_bar[1]), G_EPI_WARPS * 32);
         mbar_init(smem_u32(&ctrl->drain_bar), 1);
         ctrl->abort_flag = 0;
         mbar_fence_init();
@@ -104,6 +120,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
+        if (MODE == 2) tma_prefetch_desc(&tmOut);
     }
     tc_fence_before();
     __syncthreads();
@@ -121,27 +138,32 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
                 const int wrow = __ldg(g.tile_expert + m_tile) * g.w_rows_per_expert;
-                int b_row0, b_row1;
-                if (MODE == 1) {
-                    b_row0 = wrow + g.gate_row0 + n * 128;
-                    b_row1 = wrow + g.up_row0 + n * 128;
-                } else {
-                    b_row0 = wrow + n * G_TILE_N;
-                    b_row1 = b_row0 + 128;
-                }
+                const float* a_sc = g.a_scale_t + static_cast<size_t>(m_tile) * TILE_M;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1;
-                    if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1, abort_flag)) {
+                    if (!mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, abort_flag)) {
                         raise(ctrl, g.status, DEV_TIMEOUT_PRODUCER);
                         ok = false;
                         break;
                     }
                     const uint32_t bar = smem_u32(&ctrl->full[s]);
                     const uint32_t a_dst = smem_base + s * G_STAGE_BYTES, b_dst = a_dst + G_A_BYTES;
-                    mbar_expect_tx(bar, G_STAGE_BYTES);
-                    tma_load_2d(a_dst, &tmA, kb * G_BLOCK_K, m_tile * TILE_M, bar);
-                    tma_load_2d(b_dst, &tmB, kb * G_BLOCK_K, b_row0, bar);
-                    tma_load_2d(b_dst + G_B_BYTES / 2, &tmB, kb * G_BLOCK_K, b_row1, bar);
+                    const int k0 = kb * G_BLOCK_K;
+                    mbar_expect_tx(bar, G_STAGE_BYTES + G_SCALE_BYTES);
+                    tma_load_2d(a_dst, &tmA, k0, m_tile * TILE_M, bar);
+                    if (MODE == 1) {
+                        const int gr = wrow + g.gate_row0 + n * 128, ur = wrow + g.up_row0 + n * 128;
+                        tma_load_2d(b_dst, &tmB, k0, gr, bar);
+                        tma_load_2d(b_dst + G_B_BYTES / 4, &tmB, k0, ur, bar);
+                        tma_load_2d(b_dst + G_B_BYTES / 2, &tmB, k0, gr + 64, bar);
+                        tma_load_2d(b_dst + 3 * G_B_BYTES / 4, &tmB, k0, ur + 64, bar);
+                    } else {
+                        const int br = wrow + n * G_TILE_N;
+                        tma_load_2d(b_dst, &tmB, k0, br, bar);
+                        tma_load_2d(b_dst + G_B_BYTES / 2, &tmB, k0, br + 128, bar);
+                    }
+                    bulk_load_1d(smem_u32(scale_ring + (it % G_SCALE_RING) * TILE_M),
+                                 a_sc + static_cast<size_t>(kb) * g.row_cap, G_SCALE_BYTES, bar);
                 }
             }
             if (!ok || *abort_flag) {
@@ -179,8 +201,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
                     for (int k = 0; k < G_BLOCK_K / 32; ++k)  // 32 K-bytes per instruction: +2 in 16-B units
                         umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k > 0);
-                    umma_commit(smem_u32(&ctrl->empty[s]));
-                    umma_commit(smem_u32(&ctrl->tmem_full[b]));
+                    umma_commit(smem_u32(&ctrl->done[s]));
                 }
             }
             if (!ok || *abort_flag) {  // let issued MMAs retire before TMEM is released
@@ -192,11 +213,13 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else {
         // ---------------- epilogue warps ----------------
         reg_alloc<232>();
-        const int half = (warp - 4) >> 2;        // which half of the tile's columns
+        const int widx = warp - 4;
+        const int half = widx >> 2;              // which 128-column half of the tile
         const int quad = warp & 3;               // TMEM lane quadrant this warp may read
         const int r_in_tile = quad * 32 + lane;  // accumulator row == TMEM lane
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
         const size_t row_cap = static_cast<size_t>(g.row_cap);
+        float* amax_x = reinterpret_cast<float*>(store_stage);  // [2][2][TILE_M], GEMM1 only
         uint32_t it = 0, tile_iter = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tile_iter) {
@@ -204,9 +227,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int e = __ldg(g.tile_expert + m_tile);
             const int rows_valid = __ldg(g.tile_rows + m_tile);
             const size_t row = static_cast<size_t>(m_tile) * TILE_M + r_in_tile;
-            const float* a_sc = g.a_scale_t + row;
             const int sblocks = g.w_rows_per_expert / 128;
-            // weight-scale rows for the two 64-column (GEMM1) or the one 128-column (GEMM2) block(s)
+            // weight-scale rows of this thread's first / second 64 columns
             const float* ws0;
             const float* ws1;
             if (MODE == 1) {
@@ -216,60 +238,66 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + 2 * n + half) * num_kb;
                 ws1 = ws0;
             }
-            float acc[128];
+            uint64_t acc[64];  // 128 fp32 accumulators, two per register pair
 #pragma unroll
-            for (int j = 0; j < 128; ++j) acc[j] = 0.0f;
-            float sa = a_sc[0], s0 = __ldg(ws0), s1 = __ldg(ws1);
+            for (int j = 0; j < 64; ++j) acc[j] = 0ull;
+            float s0 = __ldg(ws0), s1 = __ldg(ws1);
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                const float f0 = sa * s0, f1 = sa * s1;
-                if (kb + 1 < num_kb) {  // next block's scales travel while we wait for the MMA
-                    sa = a_sc[static_cast<size_t>(kb + 1) * row_cap];
+                const float w0 = s0, w1 = s1;
+                if (kb + 1 < num_kb) {
                     s0 = __ldg(ws0 + kb + 1);
                     s1 = __ldg(ws1 + kb + 1);
                 }
-                const uint32_t b = it & 1, bph = (it >> 1) & 1;
-                if (!mbar_wait(smem_u32(&ctrl->tmem_full[b]), bph, abort_flag)) {
+                const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1, buf = it & 1;
+                if (!mbar_wait(smem_u32(&ctrl->done[s]), ph, abort_flag)) {
                     raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                // GEMM1: columns [64h,64h+64) are gate, [128+64h, 128+64h+64) the matching up columns.
-                // GEMM2: columns [128h, 128h+128).
-                const uint32_t col0 = b * G_TILE_N + (MODE == 1 ? 64 * half : 128 * half);
-                const uint32_t col1 = b * G_TILE_N + (MODE == 1 ? 128 + 64 * half : 128 * half + 64);
+                // The MMA of this K-block has finished, hence its stage -- A, B and the scales -- had landed.
+                const float sa =
+                    *reinterpret_cast<volatile float*>(scale_ring + (it % G_SCALE_RING) * TILE_M + r_in_tile);
+                const float f0 = sa * w0, f1 = sa * w1;
+                const uint64_t ff0 = pack2(f0, f0), ff1 = pack2(f1, f1);
+                // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
+                const uint32_t col = t_lane + buf * G_TILE_N + half * G_HALF_N;
                 float v[64];
-                tmem_ld64(t_lane + col0, v);
+                tmem_ld64(col, v);
 #pragma unroll
-                for (int j = 0; j < 64; ++j) acc[j] = fmaf(v[j], f0, acc[j]);
-                tmem_ld64(t_lane + col1, v);
+                for (int j = 0; j < 32; ++j) fma2(acc[j], pack2(v[2 * j], v[2 * j + 1]), ff0);
+                tmem_ld64(col + 64, v);
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[b]));
+                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
 #pragma unroll
-                for (int j = 0; j < 64; ++j) acc[64 + j] = fmaf(v[j], f1, acc[64 + j]);
+                for (int j = 0; j < 32; ++j) fma2(acc[32 + j], pack2(v[2 * j], v[2 * j + 1]), ff1);
             }
             if (!ok) break;
 
             if (MODE == 1) {
                 // SwiGLU on this thread's 64 columns, then the row's 128-wide amax across the two halves
+                float c[64];
                 float amax = 0.0f;
 #pragma unroll
-                for (int j = 0; j < 64; ++j) {
-                    const float gt = acc[j];
-                    const float c = __fdiv_rn(gt, 1.0f + expf(-gt)) * acc[64 + j];
-                    acc[j] = c;
-                    amax = fmaxf(amax, fabsf(c));
+                for (int j = 0; j < 32; ++j) {
+                    float g0, g1, u0, u1;
+                    unpack2(acc[j], g0, g1);
+                    unpack2(acc[32 + j], u0, u1);
+                    c[2 * j] = __fdiv_rn(g0, 1.0f + expf(-g0)) * u0;
+                    c[2 * j + 1] = __fdiv_rn(g1, 1.0f + expf(-g1)) * u1;
+                    amax = fmaxf(amax, fmaxf(fabsf(c[2 * j]), fabsf(c[2 * j + 1])));
                 }
                 const uint32_t par = tile_iter & 1;
-                ctrl->amax[par][half][r_in_tile] = amax;
+                amax_x[(par * 2 + half) * TILE_M + r_in_tile] = amax;
                 const uint32_t xbar = smem_u32(&ctrl->amax_bar[par]);
                 mbar_arrive(xbar);
                 if (!mbar_wait(xbar, (tile_iter >> 1) & 1, abort_flag)) {
                     raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
                     break;
                 }
-                amax = fmaxf(amax, *reinterpret_cast<volatile float*>(&ctrl->amax[par][half ^ 1][r_in_tile]));
+                amax = fmaxf(amax,
+                             *reinterpret_cast<volatile float*>(&amax_x[(par * 2 + (half ^ 1)) * TILE_M + r_in_tile]));
                 const float sc = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 448.0f);
                 if (r_in_tile < rows_valid) {
                     uint4* dst = reinterpret_cast<uint4*>(g.out_fp8 + row * g.out_cols + n * 128 + half * 64);
@@ -280,9 +308,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         for (int i = 0; i < 4; ++i) {
                             const int j = q * 16 + i * 4;
                             const uint32_t lo = __nv_cvt_float2_to_fp8x2(
-                                make_float2(__fdiv_rn(acc[j], sc), __fdiv_rn(acc[j + 1], sc)), __NV_SATFINITE, __NV_E4M3);
+                                make_float2(__fdiv_rn(c[j], sc), __fdiv_rn(c[j + 1], sc)), __NV_SATFINITE, __NV_E4M3);
                             const uint32_t hi = __nv_cvt_float2_to_fp8x2(
-                                make_float2(__fdiv_rn(acc[j + 2], sc), __fdiv_rn(acc[j + 3], sc)), __NV_SATFINITE,
+                                make_float2(__fdiv_rn(c[j + 2], sc), __fdiv_rn(c[j + 3], sc)), __NV_SATFINITE,
                                 __NV_E4M3);
                             w[i] = lo | (hi << 16);
                         }
@@ -291,21 +319,41 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (half == 0) g.out_scale_t[static_cast<size_t>(n) * row_cap + row] = sc;
                 }
             } else {
-                if (r_in_tile < rows_valid) {
-                    uint4* dst = reinterpret_cast<uint4*>(g.out_bf16 + row * g.out_cols + n * G_TILE_N + half * 128);
+                // bf16 rows out: each warp stages 32 rows x 32 columns (64-byte rows, 64-byte swizzle) in
+                // shared memory and one lane hands the box to the TMA engine; four passes cover 128 columns.
+                if (quad * 32 < rows_valid) {
+                    uint8_t* stage = store_stage + widx * G_STORE_WARP_BYTES;
+                    const uint32_t stage_u32 = smem_u32(stage);
+                    const int sw = (lane >> 1) & 3;
 #pragma unroll
-                    for (int q = 0; q < 16; ++q) {
-                        uint32_t w[4];
+                    for (int p = 0; p < 4; ++p) {
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const __nv_bfloat162 p = __floats2bfloat162_rn(acc[q * 8 + 2 * i], acc[q * 8 + 2 * i + 1]);
-                            w[i] = *reinterpret_cast<const uint32_t*>(&p);
+                        for (int ch = 0; ch < 4; ++ch) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                float lo, hi;
+                                unpack2(acc[p * 16 + ch * 4 + i], lo, hi);
+                                const __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
+                                w[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                            }
+                            *reinterpret_cast<uint4*>(stage + lane * 64 + ((ch ^ sw) << 4)) =
+                                make_uint4(w[0], w[1], w[2], w[3]);
                         }
-                        dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
+                        fence_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_2d(&tmOut, stage_u32, n * G_TILE_N + half * G_HALF_N + p * 32,
+                                         m_tile * TILE_M + quad * 32);
+                            bulk_commit_group();
+                            bulk_wait_read_all();  // the staging area is rewritten by the next pass
+                        }
+                        __syncwarp();
                     }
                 }
             }
         }
+        if (MODE == 2 && lane == 0) bulk_wait_all();
     }
 
     tc_fence_before();

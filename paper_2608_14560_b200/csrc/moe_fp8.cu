@@ -87,7 +87,7 @@ struct moe_fp8_handle_s {
     uint8_t* ws;
     size_t ws_bytes;
     EncodeTiledFn encode;
-    CUtensorMap tm_a1, tm_a2, tm_w13, tm_w2;
+    CUtensorMap tm_a1, tm_a2, tm_w13, tm_w2, tm_y;
     const void* w13_cached;
     const void* w2_cached;
     bool stage_timing;
@@ -102,15 +102,17 @@ int cuda_fail(moe_fp8_handle_t h, cudaError_t e) {
     return MOE_FP8_ERR_CUDA;
 }
 
-// 2-D uint8 tensor [rows, cols] (cols contiguous), box 128 bytes x 128 rows, 128-byte swizzle.
-bool encode_2d(moe_fp8_handle_t h, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols) {
+// 2-D tensor [rows, cols] (cols contiguous) of 1-byte (fp8) or 2-byte (bf16) elements for tiled TMA copies
+// with a box of box_cols x box_rows elements and the given shared-memory swizzle.
+bool encode_2d(moe_fp8_handle_t h, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, int elem_bytes,
+               uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle swizzle) {
     cuuint64_t gdim[2] = {cols, rows};
-    cuuint64_t gstride[1] = {cols};
-    cuuint32_t box[2] = {128, 128};
+    cuuint64_t gstride[1] = {cols * elem_bytes};
+    cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estride[2] = {1, 1};
-    CUresult r = h->encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), gdim, gstride, box, estride,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = h->encode(m, elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                           const_cast<void*>(base), gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -232,8 +234,11 @@ int moe_fp8_set_workspace(moe_fp8_handle_t h, void* ws, size_t bytes) {
     if (bytes < h->L.total) return MOE_FP8_ERR_NO_WORKSPACE;
     h->ws = static_cast<uint8_t*>(ws);
     h->ws_bytes = bytes;
-    if (!encode_2d(h, &h->tm_a1, h->ws + h->L.a1, h->L.row_cap, h->cfg.hidden) ||
-        !encode_2d(h, &h->tm_a2, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate)) {
+    if (!encode_2d(h, &h->tm_a1, h->ws + h->L.a1, h->L.row_cap, h->cfg.hidden, 1, 128, TILE_M,
+                   CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !encode_2d(h, &h->tm_a2, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate, 1, 128, TILE_M,
+                   CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !encode_2d(h, &h->tm_y, h->ws + h->L.y, h->L.row_cap, h->cfg.hidden, 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) {
         h->ws = nullptr;
         return cuda_fail(h, cudaErrorInvalidValue);
     }
@@ -266,8 +271,10 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     const int H = c.hidden, I = c.intermediate, EL = c.num_local_experts;
     if (w13 != h->w13_cached || w2 != h->w2_cached) {
-        if (!encode_2d(h, &h->tm_w13, w13, static_cast<uint64_t>(EL) * 2 * I, H) ||
-            !encode_2d(h, &h->tm_w2, w2, static_cast<uint64_t>(EL) * H, I))
+        // w13 is fetched in 64-row boxes (gate and up rows interleave in the B tile), w2 in 128-row boxes
+        if (!encode_2d(h, &h->tm_w13, w13, static_cast<uint64_t>(EL) * 2 * I, H, 1, 128, 64,
+                       CU_TENSOR_MAP_SWIZZLE_128B) ||
+            !encode_2d(h, &h->tm_w2, w2, static_cast<uint64_t>(EL) * H, I, 1, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B))
             return cuda_fail(h, cudaErrorInvalidValue);
         h->w13_cached = w13;
         h->w2_cached = w2;
@@ -336,7 +343,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         g.out_fp8 = a2;
         g.out_scale_t = a2_scale_t;
         g.status = status;
-        grouped_gemm_kernel<1><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a1, h->tm_w13, g);
+        grouped_gemm_kernel<1><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a1, h->tm_w13, h->tm_y, g);
         ++launches;
         mark();
     }
@@ -353,9 +360,8 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         g.tile_rows = m.tile_rows;
         g.a_scale_t = a2_scale_t;
         g.w_scale = w2_scale;
-        g.out_bf16 = y;
         g.status = status;
-        grouped_gemm_kernel<2><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a2, h->tm_w2, g);
+        grouped_gemm_kernel<2><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a2, h->tm_w2, h->tm_y, g);
         ++launches;
         mark();
     }
