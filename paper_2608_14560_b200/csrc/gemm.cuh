@@ -8,7 +8,7 @@
 //               tile (128 rows), the B tile (256 weight rows) and the 128
 //               activation scales of the block, into a 4-stage ring (128-byte
 //               swizzle) / an 8-slot scale ring, completion on mbarriers.
-//   warp 1      MMA issuer.  Four tcgen05.mma (M128 N256 K32, e4m3 -> fp32) per
+//   warps 1,2   MMA issuers (even / odd K-blocks).  Four tcgen05.mma (M128 N256 K32, e4m3 -> fp32) per
 //               K-block into one of two 256-column TMEM buffers, then ONE
 //               tcgen05.commit: the same mbarrier tells the producer that the stage
 //               is free and the epilogue that the accumulator is ready (a single
@@ -44,9 +44,10 @@ constexpr int G_THREADS = 384;                          // 4 control warps + 8 e
 constexpr int G_EPI_WARPS = 8;
 constexpr int G_STORE_WARP_BYTES = 2048;                // per-warp staging: 32 rows x 64 B (swizzled)
 constexpr int G_STORE_BYTES = G_EPI_WARPS * G_STORE_WARP_BYTES;
+constexpr int G_AMAX_BYTES = 2 * 2 * TILE_M * 4;               // GEMM1 row-amax exchange
 constexpr int G_CTRL_BYTES = 512;
 constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_SCALE_RING * G_SCALE_BYTES + G_STORE_BYTES +
-                             G_CTRL_BYTES + 1024;       // + alignment slack
+                             G_AMAX_BYTES + G_CTRL_BYTES + 1024;       // + alignment slack
 constexpr uint32_t G_TMEM_COLS = 512;
 static_assert(G_SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
 
@@ -64,6 +65,7 @@ struct GemmArgs {
     const float* w_scale;     // [E_loc, w_rows/128, num_kb]
     uint8_t* out_fp8;         // GEMM1: [row_cap, I] e4m3
     float* out_scale_t;       // GEMM1: [I/128, row_cap]
+    __nv_bfloat16* out_bf16;  // GEMM2: tile-blocked rows, see y_block_offset()
     int* status;
 };
 
@@ -72,7 +74,7 @@ struct GemmCtrl {
     uint64_t done[G_STAGES];   // the MMAs that read the stage have finished: stage free AND accumulator ready
     uint64_t tmem_empty[G_ACC_BUFS];
     uint64_t amax_bar[2];
-    uint64_t drain_bar;
+    uint64_t drain_bar[2];
     uint32_t tmem_slot;
     int abort_flag;
 };
@@ -85,7 +87,8 @@ __device__ __forceinline__ void raise(GemmCtrl* c, int* status, int code) {
 
 // MODE 1: gate/up projection + SwiGLU + re-quantisation (B tile = 4 x 64 weight rows:
 //         gate[0,64) | up[0,64) | gate[64,128) | up[64,128) of the tile's 128 columns).
-// MODE 2: down projection, bf16 rows out through TMA stores (B tile = 2 x 128 rows).
+//         tmOut describes the e4m3 output [row_cap, I] for 64-byte x 32-row TMA stores.
+// MODE 2: down projection, bf16 rows out in the tile-blocked layout (B tile = 2 x 128 rows).
 template <int MODE>
 __global__ void __launch_bounds__(G_THREADS, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -94,7 +97,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     float* scale_ring = reinterpret_cast<float*>(smem + G_STAGES * G_STAGE_BYTES);
     uint8_t* store_stage = smem + G_STAGES * G_STAGE_BYTES + G_SCALE_RING * G_SCALE_BYTES;
-    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(store_stage + G_STORE_BYTES);
+    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(store_stage + G_STORE_BYTES + G_AMAX_BYTES);
     volatile int* abort_flag = &ctrl->abort_flag;
     const uint32_t smem_base = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -109,7 +112,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         mbar_init(smem_u32(&ctrl->amax_bar[0]), G_EPI_WARPS * 32);
         mbar_init(smem_u32(&ctrl->amax_bar[1]), G_EPI_WARPS * 32);
-        mbar_init(smem_u32(&ctrl->drain_bar), 1);
+        mbar_init(smem_u32(&ctrl->drain_bar[0]), 1);
+        mbar_init(smem_u32(&ctrl->drain_bar[1]), 1);
         ctrl->abort_flag = 0;
         mbar_fence_init();
     }
@@ -120,7 +124,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == 0 && lane == 0) {
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
-        if (MODE == 2) tma_prefetch_desc(&tmOut);
+        if (MODE == 1) tma_prefetch_desc(&tmOut);
     }
     tc_fence_before();
     __syncthreads();
@@ -174,13 +178,18 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (!mbar_wait(smem_u32(&ctrl->full[j % G_STAGES]), (j / G_STAGES) & 1, &zero))
                         atomicCAS(g.status, DEV_OK, DEV_TIMEOUT_DRAIN);
             }
-        } else if (warp == 1 && lane == 0) {
-            // ---------------- MMA issuer ----------------
+        } else if ((warp == 1 || warp == 2) && lane == 0) {
+            // ---------------- MMA issuers ----------------
+            // Two threads share the issue work: warp 1 takes the even K-blocks (TMEM buffer 0), warp 2 the
+            // odd ones (buffer 1).  A commit only tracks the MMAs of its own thread, so while one thread
+            // pays for its commit and waits the other keeps the tensor pipe fed.
             const uint32_t idesc = umma_idesc_f8(TILE_M, G_TILE_N);
+            const uint32_t mine = warp - 1;
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    if ((it & 1) != mine) continue;
                     const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1;
                     const uint32_t b = it & 1, bph = (it >> 1) & 1;
                     if (!mbar_wait(smem_u32(&ctrl->tmem_empty[b]), bph ^ 1, abort_flag)) {
@@ -205,9 +214,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
             }
             if (!ok || *abort_flag) {  // let issued MMAs retire before TMEM is released
-                umma_commit(smem_u32(&ctrl->drain_bar));
+                umma_commit(smem_u32(&ctrl->drain_bar[mine]));
                 int zero = 0;
-                mbar_wait(smem_u32(&ctrl->drain_bar), 0, &zero);
+                mbar_wait(smem_u32(&ctrl->drain_bar[mine]), 0, &zero);
             }
         }
     } else {
@@ -217,9 +226,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int half = widx >> 2;              // which 128-column half of the tile
         const int quad = warp & 3;               // TMEM lane quadrant this warp may read
         const int r_in_tile = quad * 32 + lane;  // accumulator row == TMEM lane
-        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * G_HALF_N;
         const size_t row_cap = static_cast<size_t>(g.row_cap);
-        float* amax_x = reinterpret_cast<float*>(store_stage);  // [2][2][TILE_M], GEMM1 only
+        float* amax_x = reinterpret_cast<float*>(store_stage + G_STORE_BYTES);  // [2][2][TILE_M], GEMM1 only
+        uint8_t* stage = store_stage + widx * G_STORE_WARP_BYTES;
         uint32_t it = 0, tile_iter = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tile_iter) {
@@ -241,6 +251,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             uint64_t acc[64];  // 128 fp32 accumulators, two per register pair
 #pragma unroll
             for (int j = 0; j < 64; ++j) acc[j] = 0ull;
+
             float s0 = __ldg(ws0), s1 = __ldg(ws1);
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
                 const float w0 = s0, w1 = s1;
@@ -261,7 +272,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const float f0 = sa * w0, f1 = sa * w1;
                 const uint64_t ff0 = pack2(f0, f0), ff1 = pack2(f1, f1);
                 // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
-                const uint32_t col = t_lane + buf * G_TILE_N + half * G_HALF_N;
+                const uint32_t col = t_lane + buf * G_TILE_N;
                 float v[64];
                 tmem_ld64(col, v);
 #pragma unroll
@@ -274,6 +285,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 for (int j = 0; j < 32; ++j) fma2(acc[32 + j], pack2(v[2 * j], v[2 * j + 1]), ff1);
             }
             if (!ok) break;
+
+            // The staging area of this warp was handed to the TMA engine at the end of the previous tile;
+            // by now (a whole tile later) that copy has long read it, so this wait does not stall.
+            if (lane == 0) bulk_wait_read_all();
+            __syncwarp();
+            const int sw = (lane >> 1) & 3;  // 64-byte swizzle: 16-byte chunk index ^= bits 7..8 of the address
 
             if (MODE == 1) {
                 // SwiGLU on this thread's 64 columns, then the row's 128-wide amax across the two halves
@@ -299,8 +316,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 amax = fmaxf(amax,
                              *reinterpret_cast<volatile float*>(&amax_x[(par * 2 + (half ^ 1)) * TILE_M + r_in_tile]));
                 const float sc = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 448.0f);
-                if (r_in_tile < rows_valid) {
-                    uint4* dst = reinterpret_cast<uint4*>(g.out_fp8 + row * g.out_cols + n * 128 + half * 64);
+                if (quad * 32 < rows_valid) {
+                    // e4m3 rows out: 32 rows x 64 bytes per warp, staged with the 64-byte swizzle, one TMA store
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         uint32_t w[4];
@@ -314,46 +331,42 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                 __NV_E4M3);
                             w[i] = lo | (hi << 16);
                         }
-                        dst[q] = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4*>(stage + lane * 64 + ((q ^ sw) << 4)) =
+                            make_uint4(w[0], w[1], w[2], w[3]);
                     }
-                    if (half == 0) g.out_scale_t[static_cast<size_t>(n) * row_cap + row] = sc;
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmOut, smem_u32(stage), n * 128 + half * 64, m_tile * TILE_M + quad * 32);
+                        bulk_commit_group();
+                    }
+                    if (half == 0 && r_in_tile < rows_valid)
+                        g.out_scale_t[static_cast<size_t>(n) * row_cap + row] = sc;
                 }
             } else {
-                // bf16 rows out: each warp stages 32 rows x 32 columns (64-byte rows, 64-byte swizzle) in
-                // shared memory and one lane hands the box to the TMA engine; four passes cover 128 columns.
+                // bf16 rows out in a tile-blocked layout: block (row tile, column tile, half, quadrant) holds
+                // this warp's 32 rows x 128 columns as [8 column groups][32 rows][16 bf16], so every warp
+                // store instruction writes 1 KB of contiguous memory (32 bytes per lane).
                 if (quad * 32 < rows_valid) {
-                    uint8_t* stage = store_stage + widx * G_STORE_WARP_BYTES;
-                    const uint32_t stage_u32 = smem_u32(stage);
-                    const int sw = (lane >> 1) & 3;
+                    uint8_t* blk = reinterpret_cast<uint8_t*>(g.out_bf16) +
+                                   (((static_cast<size_t>(m_tile) * g.n_tiles + n) * 2 + half) * 4 + quad) * 8192 +
+                                   lane * 32;
 #pragma unroll
-                    for (int p = 0; p < 4; ++p) {
+                    for (int q = 0; q < 8; ++q) {
+                        uint32_t w[8];
 #pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                float lo, hi;
-                                unpack2(acc[p * 16 + ch * 4 + i], lo, hi);
-                                const __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
-                                w[i] = *reinterpret_cast<const uint32_t*>(&pr);
-                            }
-                            *reinterpret_cast<uint4*>(stage + lane * 64 + ((ch ^ sw) << 4)) =
-                                make_uint4(w[0], w[1], w[2], w[3]);
+                        for (int i = 0; i < 8; ++i) {
+                            float lo, hi;
+                            unpack2(acc[q * 8 + i], lo, hi);
+                            const __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
+                            w[i] = *reinterpret_cast<const uint32_t*>(&pr);
                         }
-                        fence_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            tma_store_2d(&tmOut, stage_u32, n * G_TILE_N + half * G_HALF_N + p * 32,
-                                         m_tile * TILE_M + quad * 32);
-                            bulk_commit_group();
-                            bulk_wait_read_all();  // the staging area is rewritten by the next pass
-                        }
-                        __syncwarp();
+                        st_global_v8(blk + q * 1024, w);
                     }
                 }
             }
         }
-        if (MODE == 2 && lane == 0) bulk_wait_all();
+        if (lane == 0) bulk_wait_all();
     }
 
     tc_fence_before();
@@ -362,6 +375,14 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         __syncwarp();
         tmem_dealloc(tmem_base, G_TMEM_COLS);
     }
+}
+
+// Byte offset of the 32-byte group holding columns [16*c16, 16*c16+16) of padded row r in the
+// tile-blocked bf16 output of GEMM2 (n_tiles = H / 256 column tiles).
+__host__ __device__ __forceinline__ size_t y_block_offset(int r, int c16, int n_tiles) {
+    const int m_tile = r / TILE_M, quad = (r % TILE_M) / 32, lane = r % 32;
+    const int n = c16 / 16, half = (c16 % 16) / 8, q = c16 % 8;
+    return (((static_cast<size_t>(m_tile) * n_tiles + n) * 2 + half) * 4 + quad) * 8192 + q * 1024 + lane * 32;
 }
 
 }  // namespace moe

@@ -87,7 +87,7 @@ struct moe_fp8_handle_s {
     uint8_t* ws;
     size_t ws_bytes;
     EncodeTiledFn encode;
-    CUtensorMap tm_a1, tm_a2, tm_w13, tm_w2, tm_y;
+    CUtensorMap tm_a1, tm_a2, tm_a2_store, tm_w13, tm_w2;
     const void* w13_cached;
     const void* w2_cached;
     bool stage_timing;
@@ -159,7 +159,9 @@ __global__ void export_rows_kernel(int E_loc, int I, int H, int row_cap, const i
             for (int i = threadIdx.x; i < I / 128; i += blockDim.x)
                 a2_scale_out[static_cast<size_t>(r) * (I / 128) + i] = a2_scale_t[static_cast<size_t>(i) * row_cap + p];
         if (y_out)
-            for (int i = threadIdx.x; i < H; i += blockDim.x) y_out[static_cast<size_t>(r) * H + i] = y[p * H + i];
+            for (int i = threadIdx.x; i < H; i += blockDim.x)
+                y_out[static_cast<size_t>(r) * H + i] = *reinterpret_cast<const __nv_bfloat16*>(
+                    reinterpret_cast<const uint8_t*>(y) + y_block_offset(static_cast<int>(p), i / 16, H / 256) + (i % 16) * 2);
     }
 }
 
@@ -238,7 +240,8 @@ int moe_fp8_set_workspace(moe_fp8_handle_t h, void* ws, size_t bytes) {
                    CU_TENSOR_MAP_SWIZZLE_128B) ||
         !encode_2d(h, &h->tm_a2, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate, 1, 128, TILE_M,
                    CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !encode_2d(h, &h->tm_y, h->ws + h->L.y, h->L.row_cap, h->cfg.hidden, 2, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) {
+        !encode_2d(h, &h->tm_a2_store, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate, 1, 64, 32,
+                   CU_TENSOR_MAP_SWIZZLE_64B)) {
         h->ws = nullptr;
         return cuda_fail(h, cudaErrorInvalidValue);
     }
@@ -343,7 +346,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         g.out_fp8 = a2;
         g.out_scale_t = a2_scale_t;
         g.status = status;
-        grouped_gemm_kernel<1><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a1, h->tm_w13, h->tm_y, g);
+        grouped_gemm_kernel<1><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a1, h->tm_w13, h->tm_a2_store, g);
         ++launches;
         mark();
     }
@@ -360,14 +363,16 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         g.tile_rows = m.tile_rows;
         g.a_scale_t = a2_scale_t;
         g.w_scale = w2_scale;
+        g.out_bf16 = y;
         g.status = status;
-        grouped_gemm_kernel<2><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a2, h->tm_w2, h->tm_y, g);
+        grouped_gemm_kernel<2><<<h->sm_count, G_THREADS, G_SMEM_BYTES, stream>>>(h->tm_a2, h->tm_w2, h->tm_a2_store, g);
         ++launches;
         mark();
     }
     {  // stage 4: weighted combine back to token order
         const int grid = min(T, h->sm_count * 16);
-        combine_kernel<<<grid, 256, 0, stream>>>(T, H, m.slot_to_row, topk_w, y, static_cast<__nv_bfloat16*>(out));
+        combine_kernel<<<grid, 256, 0, stream>>>(T, H, m.slot_to_row, topk_w, reinterpret_cast<const uint8_t*>(y),
+                                                 static_cast<__nv_bfloat16*>(out));
         ++launches;
         mark();
     }
