@@ -43,6 +43,7 @@ extern "C" {
 #define MOE_FP8_ERR_NO_WORKSPACE (-3)     /* workspace missing or too small */
 #define MOE_FP8_ERR_CUDA (-4)             /* a CUDA call failed; see moe_fp8_last_cuda_error */
 #define MOE_FP8_ERR_ARCH (-5)             /* current device is not compute capability 10.x */
+#define MOE_FP8_ERR_STATIC_LIMIT (-6)     /* size beyond the fixed capacity of a no-allocation entry point */
 
 /* Layer shape, fixed at creation.  Supported: num_experts = 256, n_group = 8,
  * topk_group = 4, top_k = 8 (the DeepSeek-V3 routing of stage 1); hidden a
@@ -140,6 +141,35 @@ const char* moe_fp8_stage_name(int i);
  * stage in milliseconds to host_ms[0..n) (host pointer); returns the number of
  * stages written. */
 int moe_fp8_get_stage_times(moe_fp8_handle_t h, float* host_ms, int n);
+
+/*
+ * Per-expert histogram and exclusive scan WITHOUT any caller-provided or allocated scratch (the paper has
+ * no counterpart; it exists for callers that cannot allocate).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a CUDA-graph capture or a
+ * latency-critical serving loop that must not take the allocator lock or trigger an implicit device
+ * synchronisation, or a plug-in that is handed tensors and a stream by its host framework but owns no
+ * memory pool.  Such a caller cannot size and hand over the workspace that moe_fp8_set_workspace wants, yet
+ * may still need the expert load (for capacity planning, load-balance statistics or to size its own
+ * buffers) from routing indices it already holds.
+ *
+ *   topk_idx       int32 [T, 8]  device, selected global expert ids per token (as moe_fp8_debug_export gives)
+ *   expert_count   int32 [num_local_experts]    device, out
+ *   expert_offset  int32 [num_local_experts+1]  device, out, exclusive scan of the counts
+ *
+ * The scratch (per-block partial counts) is a 64 KB array that lives in the library image on every GPU that
+ * loads it, for as long as the process runs.  Capacity: T <= MOE_FP8_STATIC_HISTOGRAM_MAX_TOKENS and
+ * num_local_experts <= 256; a larger T returns MOE_FP8_ERR_STATIC_LIMIT and nothing is enqueued.  The call
+ * makes no cudaMalloc/cudaFree and calls no allocating library routine; it only enqueues two kernels on
+ * `stream`.  The first call on each device looks up the device address of the array (a host-side query, no
+ * allocation); make that first call outside of any stream capture.  All calls share the one array and it
+ * keeps the previous call's contents: every entry a call reads is first written by that same call, so
+ * stale contents are never seen, but two calls whose kernels overlap on the GPU (different streams, or
+ * threads racing on one stream's order) would overwrite each other's partial counts -- serialise them.
+ */
+#define MOE_FP8_STATIC_HISTOGRAM_MAX_TOKENS 16384
+int moe_fp8_expert_histogram_static(int T, const int* topk_idx, int local_expert_offset, int num_local_experts,
+                                    int* expert_count, int* expert_offset, void* stream);
 
 /* CUDA error code (cudaError_t as int) of the last MOE_FP8_ERR_CUDA on this handle. */
 int moe_fp8_last_cuda_error(moe_fp8_handle_t h);

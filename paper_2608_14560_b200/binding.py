@@ -17,7 +17,7 @@ EXPORTS = (
     "moe_fp8_create", "moe_fp8_destroy", "moe_fp8_workspace_bytes", "moe_fp8_set_workspace", "moe_fp8_forward",
     "moe_fp8_forward_host", "moe_fp8_debug_export", "moe_fp8_last_cuda_error", "moe_fp8_last_launch_count",
     "moe_fp8_strerror", "moe_fp8_set_stage_timing", "moe_fp8_num_stages", "moe_fp8_stage_name",
-    "moe_fp8_get_stage_times",
+    "moe_fp8_get_stage_times", "moe_fp8_expert_histogram_static",
 )
 
 
@@ -72,6 +72,8 @@ def load_library() -> C.CDLL:
         lib.moe_fp8_stage_name.restype = C.c_char_p
         lib.moe_fp8_get_stage_times.argtypes = [vp, C.POINTER(C.c_float), C.c_int]
         lib.moe_fp8_get_stage_times.restype = C.c_int
+        lib.moe_fp8_expert_histogram_static.argtypes = [C.c_int, ip, C.c_int, C.c_int, ip, ip, vp]
+        lib.moe_fp8_expert_histogram_static.restype = C.c_int
         lib.moe_fp8_strerror.argtypes = [C.c_int]
         lib.moe_fp8_strerror.restype = C.c_char_p
         _lib = lib
@@ -80,6 +82,22 @@ def load_library() -> C.CDLL:
 
 def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+STATIC_HISTOGRAM_MAX_TOKENS = 16384
+ERR_STATIC_LIMIT = -6
+
+
+def expert_histogram_static(topk_idx: torch.Tensor, local_expert_offset: int, num_local_experts: int,
+                            expert_count: torch.Tensor, expert_offset: torch.Tensor, stream=None) -> int:
+    """moe_fp8_expert_histogram_static: per-expert counts and offsets from routing indices without any
+    workspace or allocation (for callers that may not allocate: graph capture, serving loops, plug-ins
+    without a memory pool).  The caller passes the preallocated int32 outputs; returns the C return code."""
+    lib = load_library()
+    s = torch.cuda.current_stream(topk_idx.device) if stream is None else stream
+    return int(lib.moe_fp8_expert_histogram_static(
+        int(topk_idx.shape[0]), _ptr(topk_idx), int(local_expert_offset), int(num_local_experts),
+        _ptr(expert_count), _ptr(expert_offset), C.c_void_p(s.cuda_stream)))
 
 
 class MoeFp8:

@@ -31,7 +31,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
         tmp = LIB_PATH + f".tmp{os.getpid()}"
         cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", tmp,
-               os.path.join(_CSRC, "moe_fp8.cu")]
+               os.path.join(_CSRC, "moe_fp8.cu"), os.path.join(_CSRC, "histogram_static.cu")]
         subprocess.check_call(cmd)
         os.replace(tmp, LIB_PATH)
     return LIB_PATH

@@ -177,6 +177,7 @@ const char* moe_fp8_strerror(int rc) {
         case MOE_FP8_ERR_NO_WORKSPACE: return "workspace missing or too small";
         case MOE_FP8_ERR_CUDA: return "CUDA error";
         case MOE_FP8_ERR_ARCH: return "device is not compute capability 10.x (no fallback path exists)";
+        case MOE_FP8_ERR_STATIC_LIMIT: return "size exceeds the fixed capacity of the no-allocation entry point";
         default: return "unknown error";
     }
 }
