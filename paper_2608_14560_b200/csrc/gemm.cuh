@@ -248,9 +248,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + 2 * n + half) * num_kb;
                 ws1 = ws0;
             }
-            uint64_t acc[64];  // 128 fp32 accumulators, two per register pair
+            float acc[128];
 #pragma unroll
-            for (int j = 0; j < 64; ++j) acc[j] = 0ull;
+            for (int j = 0; j < 128; ++j) acc[j] = 0.0f;
 
             float s0 = __ldg(ws0), s1 = __ldg(ws1);
             for (int kb = 0; kb < num_kb; ++kb, ++it) {
@@ -270,19 +270,18 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const float sa =
                     *reinterpret_cast<volatile float*>(scale_ring + (it % G_SCALE_RING) * TILE_M + r_in_tile);
                 const float f0 = sa * w0, f1 = sa * w1;
-                const uint64_t ff0 = pack2(f0, f0), ff1 = pack2(f1, f1);
                 // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
                 const uint32_t col = t_lane + buf * G_TILE_N;
                 float v[64];
                 tmem_ld64(col, v);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) fma2(acc[j], pack2(v[2 * j], v[2 * j + 1]), ff0);
+                for (int j = 0; j < 64; ++j) acc[j] = fmaf(v[j], f0, acc[j]);
                 tmem_ld64(col + 64, v);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
 #pragma unroll
-                for (int j = 0; j < 32; ++j) fma2(acc[32 + j], pack2(v[2 * j], v[2 * j + 1]), ff1);
+                for (int j = 0; j < 64; ++j) acc[64 + j] = fmaf(v[j], f1, acc[64 + j]);
             }
             if (!ok) break;
 
@@ -297,13 +296,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 float c[64];
                 float amax = 0.0f;
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float g0, g1, u0, u1;
-                    unpack2(acc[j], g0, g1);
-                    unpack2(acc[32 + j], u0, u1);
-                    c[2 * j] = __fdiv_rn(g0, 1.0f + expf(-g0)) * u0;
-                    c[2 * j + 1] = __fdiv_rn(g1, 1.0f + expf(-g1)) * u1;
-                    amax = fmaxf(amax, fmaxf(fabsf(c[2 * j]), fabsf(c[2 * j + 1])));
+                for (int j = 0; j < 64; ++j) {
+                    const float gt = acc[j];
+                    c[j] = __fdiv_rn(gt, 1.0f + expf(-gt)) * acc[64 + j];
+                    amax = fmaxf(amax, fabsf(c[j]));
                 }
                 const uint32_t par = tile_iter & 1;
                 amax_x[(par * 2 + half) * TILE_M + r_in_tile] = amax;
@@ -356,9 +352,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         uint32_t w[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            float lo, hi;
-                            unpack2(acc[q * 8 + i], lo, hi);
-                            const __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
+                            const __nv_bfloat162 pr = __floats2bfloat162_rn(acc[q * 16 + 2 * i], acc[q * 16 + 2 * i + 1]);
                             w[i] = *reinterpret_cast<const uint32_t*>(&pr);
                         }
                         st_global_v8(blk + q * 1024, w);
