@@ -18,7 +18,7 @@
 //               multiplied by fp32 scales before it joins the running sum.
 //   warps 4-7   epilogue of columns [0,128), warps 8-11 of columns [128,256): read
 //               the partial from TMEM, multiply by a_scale[row,kb] * w_scale[nblk,kb]
-//               with packed fp32 FMAs, accumulate in registers; at the end of the
+//               with fp32 FMAs, accumulate in registers; at the end of the
 //               tile apply the fused tail and store.
 // Scales are arbitrary fp32 (amax/448), so the power-of-two hardware block
 // scaling cannot express them; the per-K-block promotion is done on the ALUs.
