@@ -35,6 +35,12 @@ W13_BYTES_PER_EXPERT = 4096 * 7168 + 32 * 56 * 4
 W2_BYTES_PER_EXPERT = 7168 * 2048 + 56 * 16 * 4
 FP8_DATASHEET_TFLOPS = 4500.0
 HBM_DATASHEET_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the headline
+# workload (profiles/launches_dsv3_T64_E32.md), mean over the two rotating activation sets.
+NCU_TRAFFIC_BYTES = {
+    ("dsv3_T64_E32", "gemm1_swiglu_quant"): (486.1e6 + 3.9e6 + 455.8e6 + 0.8e6) / 2,
+    ("dsv3_T64_E32", "gemm2"): (239.5e6 + 2.8e6 + 224.4e6 + 2.6e6) / 2,
+}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -224,6 +230,9 @@ def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, 
         ach = kern_bytes / dom_s / 1e9
         res["roofline"] = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peak_kind} copy bandwidth"}
+    res["roofline"]["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name, dom))
+    res["roofline"]["algorithmic_per_launch"] = kern_flops if res["roofline"]["bound"] == "tensor" else kern_bytes
+    res["roofline"]["kernel_ms"] = stage_avg[dom]
     if sampler:
         res["clocks"] = sampler.result()
 
