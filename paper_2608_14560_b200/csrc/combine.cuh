@@ -17,6 +17,8 @@ __global__ void __launch_bounds__(256) combine_kernel(int T, int H, const int* _
                                                       const float* __restrict__ topk_w,
                                                       const uint8_t* __restrict__ y,
                                                       __nv_bfloat16* __restrict__ out) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int groups = H / 16, n_tiles = H / 256;
     for (int t = blockIdx.x; t < T; t += gridDim.x) {
         int rows[8];

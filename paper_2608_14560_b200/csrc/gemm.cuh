@@ -129,6 +129,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // Everything above touched only this CTA's shared and tensor memory; the tile tables, activations and
+    // scales below were written by the kernels before this one.
+    pdl_launch_dependents();
+    pdl_wait();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_slot);
     const int num_tiles = __ldg(g.num_m_tiles) * g.n_tiles;
     const int num_kb = g.num_kb;

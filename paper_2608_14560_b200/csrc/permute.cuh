@@ -10,6 +10,8 @@
 #pragma once
 #include <stdint.h>
 
+#include "ptx.cuh"
+
 namespace moe {
 
 constexpr int P_TOKENS_PER_BLOCK = 256;  // tokens handled by one block of the count/place kernels
@@ -53,6 +55,8 @@ __device__ __forceinline__ void build_block_masks(uint32_t (*mask)[P_TOKENS_PER_
 __global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) count_kernel(int T, int E_loc, int off,
                                                                    const int* __restrict__ topk_idx,
                                                                    int* __restrict__ block_hist) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ uint32_t mask[P_MAX_LOCAL][P_TOKENS_PER_BLOCK / 32];
     build_block_masks(mask, T, E_loc, off, topk_idx);
     for (int e = threadIdx.x; e < E_loc; e += blockDim.x) {
@@ -65,6 +69,8 @@ __global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) count_kernel(int T, int E_
 
 // One block.  Thread e owns local expert e.
 __global__ void __launch_bounds__(P_MAX_LOCAL) scan_kernel(int nblk, int E_loc, PermuteMeta m) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ int s_cnt[P_MAX_LOCAL + 1];
     __shared__ int s_pad[P_MAX_LOCAL + 1];
     const int e = threadIdx.x;
@@ -112,6 +118,8 @@ __global__ void __launch_bounds__(P_MAX_LOCAL) scan_kernel(int nblk, int E_loc, 
 __global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) place_kernel(int T, int E_loc, int off, int row_cap,
                                                                    const int* __restrict__ topk_idx, PermuteMeta m,
                                                                    int* __restrict__ status) {
+    pdl_launch_dependents();
+    pdl_wait();
     __shared__ uint32_t mask[P_MAX_LOCAL][P_TOKENS_PER_BLOCK / 32];
     build_block_masks(mask, T, E_loc, off, topk_idx);
     const int t = blockIdx.x * P_TOKENS_PER_BLOCK + threadIdx.x;
@@ -146,6 +154,8 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(int H, int row_cap, in
                                                           const uint8_t* __restrict__ hidden,
                                                           const float* __restrict__ hidden_scale, PermuteMeta m,
                                                           uint8_t* __restrict__ a1, float* __restrict__ a1_scale_t) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int warp = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int nwarps = gridDim.x * (blockDim.x >> 5);

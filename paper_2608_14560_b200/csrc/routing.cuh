@@ -9,6 +9,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include "ptx.cuh"
+
 namespace moe {
 
 constexpr int R_EXPERTS = 256;  // global experts
@@ -50,6 +52,8 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 __global__ void __launch_bounds__(256) route_topk_kernel(int T, const float* __restrict__ logits,
                                                          const __nv_bfloat16* __restrict__ bias, float scaling,
                                                          int* __restrict__ topk_idx, float* __restrict__ topk_w) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int warps_per_block = blockDim.x >> 5;
     const int warp0 = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
