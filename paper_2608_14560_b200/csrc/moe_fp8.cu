@@ -155,6 +155,9 @@ PermuteMeta meta_of(moe_fp8_handle_t h) {
 }
 
 constexpr int PDL_MAX_TOKENS = 2048;
+// One block routes one token per warp: measured faster than the four separate kernels up to 32 tokens only.
+constexpr int FUSED_ROUTE_MAX_TOKENS = 32;
+static_assert(FUSED_ROUTE_MAX_TOKENS <= P_TOKENS_PER_BLOCK, "the fused kernel handles one block of tokens");
 constexpr int NUM_STAGES = 8;
 const char* const STAGE_NAMES[NUM_STAGES] = {"route_topk", "count", "scan", "place", "gather_rows",
                                              "gemm1_swiglu_quant", "gemm2", "combine"};
@@ -329,14 +332,24 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     h->stage_times_valid = false;
     mark();
 
-    {  // stage 1: routing
-        const int grid = min((T + 7) / 8, h->sm_count * 8);
-        launch(route_topk_kernel, grid, 256, 0, stream, false, T, router_logits,
-               static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w);
+    if (T <= FUSED_ROUTE_MAX_TOKENS) {  // stages 1-2 without the gather in one block (one warp per token)
+        launch(route_permute_small_kernel, 1, P_FUSED_THREADS, 0, stream, false, T, EL, local_expert_offset, row_cap,
+               router_logits, static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w, m,
+               status);
         ++launches;
         mark();
-    }
-    {  // stage 2: histogram, scan, placement, gather
+        mark();
+        mark();
+        mark();
+    } else {
+        {  // stage 1: routing
+            const int grid = min((T + 7) / 8, h->sm_count * 8);
+            launch(route_topk_kernel, grid, 256, 0, stream, false, T, router_logits,
+                   static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w);
+            ++launches;
+            mark();
+        }
+        // stage 2: histogram, scan, placement
         launch(count_kernel, nblk, P_TOKENS_PER_BLOCK, 0, stream, pdl, T, EL, local_expert_offset,
                static_cast<const int*>(topk_idx), m.block_hist);
         mark();
@@ -345,11 +358,14 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         launch(place_kernel, nblk, P_TOKENS_PER_BLOCK, 0, stream, pdl, T, EL, local_expert_offset, row_cap,
                static_cast<const int*>(topk_idx), m, status);
         mark();
+        launches += 3;
+    }
+    {  // stage 2, continued: gather
         const long long row_bound = static_cast<long long>(T) * 8 + static_cast<long long>(EL) * (TILE_M - 1);
         const int grid = static_cast<int>(std::min<long long>((row_bound + 7) / 8, h->sm_count * 8LL));
         launch(gather_rows_kernel, grid, 256, 0, stream, pdl, H, row_cap, c.hidden_scale_layout, T,
                static_cast<const uint8_t*>(hidden_fp8), hidden_scale, m, a1, a1_scale_t);
-        launches += 4;
+        ++launches;
         mark();
     }
     {  // stage 3a: GEMM1 + SwiGLU + re-quantisation

@@ -48,7 +48,99 @@ __device__ __forceinline__ uint32_t order_key(float f) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Lane l owns experts 8l .. 8l+7, so a group of 32 experts is 4 neighbouring lanes.
+// Bias of the 8 experts a lane owns (lane l owns experts 8l .. 8l+7, so a group of 32 experts is 4
+// neighbouring lanes), bf16 -> fp32.
+__device__ __forceinline__ void load_bias8(const __nv_bfloat16* __restrict__ bias, int lane, float (&bias_f)[8]) {
+    const uint4 braw = reinterpret_cast<const uint4*>(bias)[lane];
+    const uint32_t w[4] = {braw.x, braw.y, braw.z, braw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        bias_f[2 * i] = __uint_as_float(w[i] << 16);
+        bias_f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+// Routes token t with one warp.  Lane j < 8 returns the j-th selected expert and its weight.
+__device__ __forceinline__ void route_token(int t, int lane, const float* __restrict__ logits,
+                                            const float (&bias_f)[8], float scaling, int& my_idx, float& my_w) {
+    const float4* row = reinterpret_cast<const float4*>(logits + static_cast<size_t>(t) * R_EXPERTS);
+    const float4 x0 = __ldg(row + 2 * lane), x1 = __ldg(row + 2 * lane + 1);
+    const float x[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+    float sig[8], b[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        sig[i] = sigmoid_fixed(x[i]);
+        b[i] = __fadd_rn(sig[i], bias_f[i]);
+    }
+    // two largest biased scores of my 8, then of the 4 lanes of my group
+    float m1 = fmaxf(b[0], b[1]), m2 = fminf(b[0], b[1]);
+#pragma unroll
+    for (int i = 2; i < 8; ++i) {
+        m2 = fmaxf(m2, fminf(m1, b[i]));
+        m1 = fmaxf(m1, b[i]);
+    }
+#pragma unroll
+    for (int d = 1; d <= 2; d <<= 1) {
+        const float o1 = __shfl_xor_sync(0xffffffffu, m1, d);
+        const float o2 = __shfl_xor_sync(0xffffffffu, m2, d);
+        m2 = fmaxf(fminf(m1, o1), fmaxf(m2, o2));
+        m1 = fmaxf(m1, o1);
+    }
+    const float gs = __fadd_rn(m1, m2);
+    // rank of my group among the 8 (ties to the smaller group index)
+    const int g = lane >> 2;
+    int better = 0;
+#pragma unroll
+    for (int o = 0; o < R_GROUPS; ++o) {
+        const float v = __shfl_sync(0xffffffffu, gs, o * 4);
+        better += (v > gs) || (v == gs && o < g);
+    }
+    const bool kept = better < R_TOPK_GROUP;
+
+    // 8 rounds of warp arg-max over the kept experts (ties to the smaller index)
+    uint32_t key[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) key[i] = kept ? order_key(b[i]) : 0u;
+    int sel_idx[R_TOPK];
+    float sel_sig[R_TOPK];
+#pragma unroll
+    for (int j = 0; j < R_TOPK; ++j) {
+        uint32_t bk = key[0];
+        int bi = 0;
+#pragma unroll
+        for (int i = 1; i < 8; ++i)
+            if (key[i] > bk) {
+                bk = key[i];
+                bi = i;
+            }
+        const uint32_t wk = __reduce_max_sync(0xffffffffu, bk);
+        const uint32_t cand = (bk == wk) ? static_cast<uint32_t>(lane * 8 + bi) : 0xffffffffu;
+        const int win = static_cast<int>(__reduce_min_sync(0xffffffffu, cand));
+        float s = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (i == (win & 7)) s = sig[i];
+        sel_sig[j] = __shfl_sync(0xffffffffu, s, win >> 3);
+        sel_idx[j] = win;
+        if (lane == (win >> 3)) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (i == (win & 7)) key[i] = 0u;
+        }
+    }
+    float den = 0.0f;
+#pragma unroll
+    for (int j = 0; j < R_TOPK; ++j) den = __fadd_rn(den, sel_sig[j]);
+    my_idx = 0;
+    my_w = 0.0f;
+#pragma unroll
+    for (int j = 0; j < R_TOPK; ++j)
+        if (lane == j) {
+            my_idx = sel_idx[j];
+            my_w = __fmul_rn(__fdiv_rn(sel_sig[j], den), scaling);
+        }
+}
+
 __global__ void __launch_bounds__(256) route_topk_kernel(int T, const float* __restrict__ logits,
                                                          const __nv_bfloat16* __restrict__ bias, float scaling,
                                                          int* __restrict__ topk_idx, float* __restrict__ topk_w) {
@@ -58,95 +150,12 @@ __global__ void __launch_bounds__(256) route_topk_kernel(int T, const float* __r
     const int warps_per_block = blockDim.x >> 5;
     const int warp0 = blockIdx.x * warps_per_block + (threadIdx.x >> 5);
     const int nwarps = gridDim.x * warps_per_block;
-
     float bias_f[8];
-    {
-        const uint4 braw = reinterpret_cast<const uint4*>(bias)[lane];
-        const uint32_t w[4] = {braw.x, braw.y, braw.z, braw.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            bias_f[2 * i] = __uint_as_float(w[i] << 16);
-            bias_f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-        }
-    }
-
+    load_bias8(bias, lane, bias_f);
     for (int t = warp0; t < T; t += nwarps) {
-        const float4* row = reinterpret_cast<const float4*>(logits + static_cast<size_t>(t) * R_EXPERTS);
-        const float4 x0 = __ldg(row + 2 * lane), x1 = __ldg(row + 2 * lane + 1);
-        const float x[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-        float sig[8], b[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            sig[i] = sigmoid_fixed(x[i]);
-            b[i] = __fadd_rn(sig[i], bias_f[i]);
-        }
-        // two largest biased scores of my 8, then of the 4 lanes of my group
-        float m1 = fmaxf(b[0], b[1]), m2 = fminf(b[0], b[1]);
-#pragma unroll
-        for (int i = 2; i < 8; ++i) {
-            m2 = fmaxf(m2, fminf(m1, b[i]));
-            m1 = fmaxf(m1, b[i]);
-        }
-#pragma unroll
-        for (int d = 1; d <= 2; d <<= 1) {
-            const float o1 = __shfl_xor_sync(0xffffffffu, m1, d);
-            const float o2 = __shfl_xor_sync(0xffffffffu, m2, d);
-            m2 = fmaxf(fminf(m1, o1), fmaxf(m2, o2));
-            m1 = fmaxf(m1, o1);
-        }
-        const float gs = __fadd_rn(m1, m2);
-        // rank of my group among the 8 (ties to the smaller group index)
-        const int g = lane >> 2;
-        int better = 0;
-#pragma unroll
-        for (int o = 0; o < R_GROUPS; ++o) {
-            const float v = __shfl_sync(0xffffffffu, gs, o * 4);
-            better += (v > gs) || (v == gs && o < g);
-        }
-        const bool kept = better < R_TOPK_GROUP;
-
-        // 8 rounds of warp arg-max over the kept experts (ties to the smaller index)
-        uint32_t key[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) key[i] = kept ? order_key(b[i]) : 0u;
-        int sel_idx[R_TOPK];
-        float sel_sig[R_TOPK];
-#pragma unroll
-        for (int j = 0; j < R_TOPK; ++j) {
-            uint32_t bk = key[0];
-            int bi = 0;
-#pragma unroll
-            for (int i = 1; i < 8; ++i)
-                if (key[i] > bk) {
-                    bk = key[i];
-                    bi = i;
-                }
-            const uint32_t wk = __reduce_max_sync(0xffffffffu, bk);
-            const uint32_t cand = (bk == wk) ? static_cast<uint32_t>(lane * 8 + bi) : 0xffffffffu;
-            const int win = static_cast<int>(__reduce_min_sync(0xffffffffu, cand));
-            float s = 0.0f;
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (i == (win & 7)) s = sig[i];
-            sel_sig[j] = __shfl_sync(0xffffffffu, s, win >> 3);
-            sel_idx[j] = win;
-            if (lane == (win >> 3)) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (i == (win & 7)) key[i] = 0u;
-            }
-        }
-        float den = 0.0f;
-#pragma unroll
-        for (int j = 0; j < R_TOPK; ++j) den = __fadd_rn(den, sel_sig[j]);
-        int my_idx = 0;
-        float my_w = 0.0f;
-#pragma unroll
-        for (int j = 0; j < R_TOPK; ++j)
-            if (lane == j) {
-                my_idx = sel_idx[j];
-                my_w = __fmul_rn(__fdiv_rn(sel_sig[j], den), scaling);
-            }
+        int my_idx;
+        float my_w;
+        route_token(t, lane, logits, bias_f, scaling, my_idx, my_w);
         if (lane < R_TOPK) {
             topk_idx[static_cast<size_t>(t) * R_TOPK + lane] = my_idx;
             topk_w[static_cast<size_t>(t) * R_TOPK + lane] = my_w;

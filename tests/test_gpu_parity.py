@@ -23,7 +23,7 @@ def _wl(tokens, dims=SMALL, seed=0, **kw):
 
 
 # ---- small layer, every token compared ------------------------------------
-@pytest.mark.parametrize("tokens", [1, 7, 130, 1000])
+@pytest.mark.parametrize("tokens", [1, 7, 32, 33, 130, 1000])
 def test_small_layer_all_tokens(cuda_device, tokens):
     st = run_and_compare(_wl(tokens, seed=tokens), cuda_device)
     assert st["frac"] >= 0.995
