@@ -271,8 +271,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
                 tc_fence_after();
                 // The MMA of this K-block has finished, hence its stage -- A, B and the scales -- had landed.
-                const float sa =
-                    *reinterpret_cast<volatile float*>(scale_ring + (it % G_SCALE_RING) * TILE_M + r_in_tile);
+                const float sa = ld_shared_f32(scale_ring + (it % G_SCALE_RING) * TILE_M + r_in_tile);
                 const float f0 = sa * w0, f1 = sa * w1;
                 // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
                 const uint32_t col = t_lane + buf * G_TILE_N;
