@@ -272,17 +272,23 @@ def oracle_sample_tokens(wl, budget_slots=400):
     return np.arange(n, dtype=np.int32)
 
 
-def oracle_baseline(wl, host, repeats=1):
+def oracle_baseline(wl, host, min_seconds=10.0):
+    """The oracle as it stands, one thread, on a bounded token sample, repeated until ~10 s of CPU work."""
     import oracle
     d = wl.dims
     tokens = oracle_sample_tokens(wl)
     t0 = time.perf_counter()
-    for _ in range(repeats):
+    reps = 0
+    while True:
         oracle.forward(host, d.n_group, d.topk_group, d.top_k, tokens=tokens)
-    dt = (time.perf_counter() - t0) / repeats
+        reps += 1
+        if time.perf_counter() - t0 >= min_seconds or reps >= 64:
+            break
+    total = time.perf_counter() - t0
+    dt = total / reps
     return {"value": len(tokens) / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
             "sample": f"first {len(tokens)} of {wl.tokens} tokens of {wl.name} (routing on all tokens), "
-                      f"single thread, {dt:.2f} s", "host_cores": os.cpu_count()}
+                      f"single thread, {reps} pass(es), {total:.1f} s in total", "host_cores": os.cpu_count()}
 
 
 def run_reference(args, wl):
@@ -313,7 +319,7 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=1, help="index into the five benchmark workloads (headline)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
