@@ -196,21 +196,23 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if ((it & 1) != mine) continue;
                     const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1;
                     const uint32_t b = it & 1, bph = (it >> 1) & 1;
-                    if (!mbar_wait(smem_u32(&ctrl->tmem_empty[b]), bph ^ 1, abort_flag)) {
-                        raise(ctrl, g.status, DEV_TIMEOUT_MMA_TMEM);
-                        ok = false;
-                        break;
-                    }
+                    // The stage has normally landed long before the accumulator is handed back, so that
+                    // wait comes first and only the hand-over itself is left on the critical path.
+                    const uint32_t a_addr = smem_base + s * G_STAGE_BYTES;
+                    const uint64_t a_desc = umma_desc_sw128(a_addr);
+                    const uint64_t b_desc = umma_desc_sw128(a_addr + G_A_BYTES);
+                    const uint32_t d_tmem = tmem_base + b * G_TILE_N;
                     if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag)) {
                         raise(ctrl, g.status, DEV_TIMEOUT_MMA_SMEM);
                         ok = false;
                         break;
                     }
+                    if (!mbar_wait(smem_u32(&ctrl->tmem_empty[b]), bph ^ 1, abort_flag)) {
+                        raise(ctrl, g.status, DEV_TIMEOUT_MMA_TMEM);
+                        ok = false;
+                        break;
+                    }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_base + s * G_STAGE_BYTES;
-                    const uint64_t a_desc = umma_desc_sw128(a_addr);
-                    const uint64_t b_desc = umma_desc_sw128(a_addr + G_A_BYTES);
-                    const uint32_t d_tmem = tmem_base + b * G_TILE_N;
 #pragma unroll
                     for (int k = 0; k < G_BLOCK_K / 32; ++k)  // 32 K-bytes per instruction: +2 in 16-B units
                         umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k > 0);
@@ -271,6 +273,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
                 tc_fence_after();
                 // The MMA of this K-block has finished, hence its stage -- A, B and the scales -- had landed.
+                // (Waiting on full[s] here instead, to fetch the scale earlier, would be wrong: this warp may
+                // be lapped by a whole phase of that barrier, and a parity wait cannot tell the difference.)
                 const float sa = ld_shared_f32(scale_ring + (it % G_SCALE_RING) * TILE_M + r_in_tile);
                 const float f0 = sa * w0, f1 = sa * w1;
                 // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
