@@ -304,8 +304,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 float amax = 0.0f;
 #pragma unroll
                 for (int j = 0; j < 64; ++j) {
+                    // silu(g) * u with the hardware exp2 and reciprocal approximations (a few ulp): the
+                    // tile's tail runs while the tensor pipe idles, so its instruction count matters.
                     const float gt = acc[j];
-                    c[j] = __fdiv_rn(gt, 1.0f + expf(-gt)) * acc[64 + j];
+                    c[j] = __fdividef(gt, 1.0f + __expf(-gt)) * acc[64 + j];
                     amax = fmaxf(amax, fabsf(c[j]));
                 }
                 const uint32_t par = tile_iter & 1;
@@ -319,6 +321,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 amax = fmaxf(amax,
                              *reinterpret_cast<volatile float*>(&amax_x[(par * 2 + (half ^ 1)) * TILE_M + r_in_tile]));
                 const float sc = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 448.0f);
+                const float inv_sc = __frcp_rn(sc);
                 if (quad * 32 < rows_valid) {
                     // e4m3 rows out: 32 rows x 64 bytes per warp, staged with the 64-byte swizzle, one TMA store
 #pragma unroll
@@ -328,10 +331,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         for (int i = 0; i < 4; ++i) {
                             const int j = q * 16 + i * 4;
                             const uint32_t lo = __nv_cvt_float2_to_fp8x2(
-                                make_float2(__fdiv_rn(c[j], sc), __fdiv_rn(c[j + 1], sc)), __NV_SATFINITE, __NV_E4M3);
+                                make_float2(c[j] * inv_sc, c[j + 1] * inv_sc), __NV_SATFINITE, __NV_E4M3);
                             const uint32_t hi = __nv_cvt_float2_to_fp8x2(
-                                make_float2(__fdiv_rn(c[j + 2], sc), __fdiv_rn(c[j + 3], sc)), __NV_SATFINITE,
-                                __NV_E4M3);
+                                make_float2(c[j + 2] * inv_sc, c[j + 3] * inv_sc), __NV_SATFINITE, __NV_E4M3);
                             w[i] = lo | (hi << 16);
                         }
                         *reinterpret_cast<uint4*>(stage + lane * 64 + ((q ^ sw) << 4)) =
