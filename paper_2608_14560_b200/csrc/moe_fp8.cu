@@ -61,7 +61,7 @@ WsLayout make_layout(const moe_fp8_config& c) {
     L.slot_to_row = take(slots * 4);
     L.row_to_slot = take(slots * 4);
     L.row_token = take(rc * 4);
-    L.status = take(4);
+    L.status = take(8);  // device status word, then the ticket counter of route_permute_kernel
     L.a1 = take(rc * H);
     L.a1_scale_t = take(rc * (H / 128) * 4);
     L.a2 = take(rc * I);
@@ -233,6 +233,9 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
     e = cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
     if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
+    e = cudaFuncSetAttribute(route_permute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(route_permute_smem_bytes(P_TAIL_MAX_TOKENS, P_MAX_LOCAL)));
+    if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
 
     moe_fp8_handle_s* h = new (std::nothrow) moe_fp8_handle_s();
     if (!h) return MOE_FP8_ERR_BAD_ARG;
@@ -323,7 +326,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     // next kernel cost the running GEMM about 6 %, so it is limited to the launch-latency-bound regime.
     const bool pdl = !h->stage_timing && T <= PDL_MAX_TOKENS;
 
-    cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), stream);
+    cudaError_t e = cudaMemsetAsync(status, 0, 2 * sizeof(int), stream);  // status and ticket
     if (e != cudaSuccess) return cuda_fail(h, e);
     int ev_i = 0;
     auto mark = [&]() {
@@ -336,6 +339,16 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         launch(route_permute_small_kernel, 1, P_FUSED_THREADS, 0, stream, false, T, EL, local_expert_offset, row_cap,
                router_logits, static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w, m,
                status);
+        ++launches;
+        mark();
+        mark();
+        mark();
+        mark();
+    } else if (T <= P_TAIL_MAX_TOKENS) {  // routing in parallel blocks, the last one to finish does stage 2
+        const int grid = min((T + 7) / 8, h->sm_count * 8);
+        launch(route_permute_kernel, grid, P_TAIL_THREADS, route_permute_smem_bytes(T, EL), stream, false, T, EL,
+               local_expert_offset, row_cap, router_logits, static_cast<const __nv_bfloat16*>(routing_bias),
+               scaling_factor, topk_idx, topk_w, m, status + 1, status);
         ++launches;
         mark();
         mark();

@@ -244,6 +244,134 @@ __global__ void __launch_bounds__(P_FUSED_THREADS) route_permute_small_kernel(
     }
 }
 
+// Batches up to P_TAIL_MAX_TOKENS: routing in parallel blocks (one warp per token), then the block that
+// finishes last -- found with a ticket counter, nobody waits -- builds histogram, scan and placement for all
+// tokens on its own.  One launch instead of four; same arithmetic and outputs as route_topk_kernel +
+// count_kernel + scan_kernel + place_kernel.  `ticket` must be zero at launch; the last block leaves it zero.
+// Dynamic shared memory: E_loc * ceil(T/32) words of masks, then as many 16-bit prefix counts.
+constexpr int P_TAIL_MAX_TOKENS = 512;   // measured faster than the four kernels up to here, slower at 1024
+constexpr int P_TAIL_THREADS = 256;
+__host__ __device__ constexpr size_t route_permute_smem_bytes(int T, int E_loc) {
+    return static_cast<size_t>(E_loc) * ((T + 31) / 32) * 6;
+}
+__global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
+    int T, int E_loc, int off, int row_cap, const float* __restrict__ logits, const __nv_bfloat16* __restrict__ bias,
+    float scaling, int* __restrict__ topk_idx, float* __restrict__ topk_w, PermuteMeta m, int* __restrict__ ticket,
+    int* __restrict__ status) {
+    pdl_launch_dependents();
+    pdl_wait();
+    extern __shared__ uint32_t dyn_smem[];
+    __shared__ int s_cnt[P_MAX_LOCAL + 1];
+    __shared__ int s_pad[P_MAX_LOCAL + 1];
+    __shared__ int s_last;
+    const int tid = threadIdx.x, lane = tid & 31;
+    {   // stage 1: one warp per token
+        const int warps_per_block = blockDim.x >> 5;
+        const int nwarps = gridDim.x * warps_per_block;
+        float bias_f[8];
+        load_bias8(bias, lane, bias_f);
+        for (int t = blockIdx.x * warps_per_block + (tid >> 5); t < T; t += nwarps) {
+            int my_idx;
+            float my_w;
+            route_token(t, lane, logits, bias_f, scaling, my_idx, my_w);
+            if (lane < R_TOPK) {
+                topk_idx[static_cast<size_t>(t) * R_TOPK + lane] = my_idx;
+                topk_w[static_cast<size_t>(t) * R_TOPK + lane] = my_w;
+            }
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const int n = atomicAdd(ticket, 1);
+        s_last = (n == static_cast<int>(gridDim.x) - 1);
+        if (s_last) *ticket = 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    // stage 2 for all tokens, in this block.  Bit t of mask[e] says: token t routes to local expert e.
+    const int W = (T + 31) / 32;
+    uint32_t* mask = dyn_smem;                                             // [E_loc][W]
+    uint16_t* pre = reinterpret_cast<uint16_t*>(dyn_smem + E_loc * W);     // [E_loc][W] tokens of e below word w
+    for (int i = tid; i < E_loc * W; i += blockDim.x) mask[i] = 0u;
+    __syncthreads();
+    for (int t = tid; t < T; t += blockDim.x) {
+        const int4 a = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t);
+        const int4 b = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t + 1);
+        const int ids[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int e = ids[j] - off;
+            if (e >= 0 && e < E_loc) atomicOr(&mask[e * W + (t >> 5)], 1u << (t & 31));
+        }
+    }
+    __syncthreads();
+    int total = 0;
+    for (int e = tid; e < P_MAX_LOCAL; e += blockDim.x) {
+        total = 0;
+        if (e < E_loc)
+            for (int w = 0; w < W; ++w) {
+                pre[e * W + w] = static_cast<uint16_t>(total);
+                total += __popc(mask[e * W + w]);
+            }
+        s_cnt[e] = total;
+        s_pad[e] = (total + TILE_M - 1) / TILE_M * TILE_M;
+    }
+    __syncthreads();
+    if (tid == 0) {  // 256 entries: a serial scan is a few hundred cycles
+        int a = 0, p = 0;
+        for (int i = 0; i < E_loc; ++i) {
+            const int c = s_cnt[i], q = s_pad[i];
+            s_cnt[i] = a;
+            s_pad[i] = p;
+            a += c;
+            p += q;
+        }
+        s_cnt[E_loc] = a;
+        s_pad[E_loc] = p;
+        *m.num_m_tiles = p / TILE_M;
+        m.expert_offset[E_loc] = a;
+        m.padded_offset[E_loc] = p;
+    }
+    __syncthreads();
+    for (int e = tid; e < E_loc; e += blockDim.x) {  // blockDim == P_MAX_LOCAL: `total` is still expert e's count
+        m.expert_count[e] = total;
+        m.expert_offset[e] = s_cnt[e];
+        m.padded_offset[e] = s_pad[e];
+        const int t0 = s_pad[e] / TILE_M;
+        for (int i = 0; i * TILE_M < total; ++i) {
+            m.tile_expert[t0 + i] = e;
+            m.tile_rows[t0 + i] = min(TILE_M, total - i * TILE_M);
+        }
+    }
+    for (int t = tid; t < T; t += blockDim.x) {
+        const int4 a = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t);
+        const int4 b = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t + 1);
+        const int ids[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        const int word = t >> 5, bit = t & 31;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int e = ids[j] - off;
+            int prow = -1;
+            if (e >= 0 && e < E_loc) {
+                const int rank = pre[e * W + word] + __popc(mask[e * W + word] & ((1u << bit) - 1u));
+                prow = s_pad[e] + rank;
+                if (prow < 0 || prow >= row_cap) {
+                    atomicExch(status, DEV_BAD_ROW);
+                    prow = -1;
+                } else {
+                    m.row_to_slot[s_cnt[e] + rank] = t * 8 + j;
+                    m.row_token[prow] = t;
+                }
+            }
+            m.slot_to_row[t * 8 + j] = prow;
+        }
+    }
+}
+static_assert(P_TAIL_THREADS == P_MAX_LOCAL, "the tail keeps one expert's count per thread");
+
 // One warp per padded row: copy the token's FP8 row (K bytes) and write its
 // K/128 scales transposed ([K/128, row_cap]) so the GEMM epilogue reads them
 // coalesced across the rows of a tile.  Rows past an expert's count are padding
