@@ -38,8 +38,8 @@ HBM_DATASHEET_GBS = 8000.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the headline
 # workload (profiles/launches_dsv3_T64_E32.md), mean over the two rotating activation sets.
 NCU_TRAFFIC_BYTES = {
-    ("dsv3_T64_E32", "gemm1_swiglu_quant"): (486.1e6 + 3.9e6 + 455.8e6 + 0.8e6) / 2,
-    ("dsv3_T64_E32", "gemm2"): (239.5e6 + 2.8e6 + 224.4e6 + 2.6e6) / 2,
+    ("dsv3_T64_E32", "gemm1_swiglu_quant"): (486.1e6 + 4.4e6 + 455.7e6 + 0.7e6) / 2,
+    ("dsv3_T64_E32", "gemm2"): (239.5e6 + 3.2e6 + 224.5e6 + 2.6e6) / 2,
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
