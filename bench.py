@@ -339,7 +339,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override T of the chosen workload (profiling runs)")
     ap.add_argument("--paper-points", default="7,54,14107",
-                    help="token counts the paper quotes a latency for (Section 5.2, one per batch-size regime); "
+                    help="token counts the paper quotes a latency for (its table of workload regimes: short / median / long); "
                          "timed on the 32-local-expert layer and reported under 'paper_points' ('' = none)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()

@@ -129,6 +129,28 @@ def test_host_entry_point_matches_device_entry_point(cuda_device):
     eng.close()
 
 
+def test_forward_on_a_side_stream_and_after_a_change_of_weights(cuda_device):
+    # the forward is enqueued on the caller's current stream; the TMA descriptors of the weights are cached
+    # per pointer pair and must be rebuilt when other weight tensors are passed
+    wl = _wl(150, seed=21)
+    inp_a = syn.make_inputs(wl, cuda_device)
+    inp_b = syn.make_inputs(_wl(150, seed=22), cuda_device)
+    fresh = make_engine(wl, cuda_device)
+    want_b = fresh.forward(inp_b).clone()
+    fresh.close()
+    eng = make_engine(wl, cuda_device)
+    side = torch.cuda.Stream(device=cuda_device)
+    side.wait_stream(torch.cuda.current_stream(cuda_device))
+    with torch.cuda.stream(side):
+        eng.forward(inp_a)
+        got_b = eng.forward(inp_b).clone()
+    side.synchronize()
+    assert eng.status() == 0
+    assert torch.equal(want_b.view(torch.int16), got_b.view(torch.int16))
+    run_and_compare(wl, cuda_device, inp=inp_a, eng=eng)
+    eng.close()
+
+
 # ---- the five benchmark workloads at full size -----------------------------
 def _sample(T, n, seed):
     if T <= n:
@@ -140,6 +162,17 @@ def _sample(T, n, seed):
 def test_benchmark_workloads_32_local_experts(cuda_device, cfg, n_sample):
     wl = syn.CONFIGS[cfg]
     st = run_and_compare(wl, cuda_device, sample_tokens=_sample(wl.tokens, n_sample, cfg))
+    print(wl.name, st)
+
+
+@pytest.mark.parametrize("tokens,n_sample", [(7, 7), (54, 54), (14107, 32)])
+def test_token_counts_quoted_in_the_paper(cuda_device, tokens, n_sample):
+    # the paper's table of workload regimes (short / median / long) quotes one latency each for T = 7, 54 and
+    # 14107 tokens with 32 local experts
+    base = syn.CONFIGS[1]
+    wl = syn.Workload(f"dsv3_T{tokens}_E32", tokens, base.dims, base.seed, base.local_expert_offset,
+                      base.scaling_factor, base.skew)
+    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(tokens, n_sample, tokens))
     print(wl.name, st)
 
 
