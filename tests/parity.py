@@ -101,21 +101,28 @@ def run_and_compare(wl: syn.Workload, device, inp=None, sample_tokens=None, chec
     if check_rows and S > 0:
         # re-quantised SwiGLU rows of a few slots against the oracle's own intermediate
         rows = np.unique(np.linspace(0, S - 1, min(S, 24)).astype(np.int64))
+        yrows = dict(zip(rows.tolist(), dbg["y_rows"][torch.as_tensor(rows, device=dbg["y_rows"].device)].float().cpu().numpy()))
         a2 = dbg["a2_fp8"].cpu().numpy()
         a2s = dbg["a2_scale"].cpu().numpy()
-        mism = tot = 0
+        mism = tot = y_bad = y_tot = 0
         for r in rows:
             slot = int(perm["row_to_slot"][r])
             t, j = divmod(slot, d.top_k)
             e = int(ridx[t, j]) - int(inp["local_expert_offset"])
             xs = host["hidden_scale"][:, t] if scale_layout else host["hidden_scale"][t]
-            _, cq, cs = oracle.mlp_row(host["hidden_fp8"][t], xs, host["w13"][e], host["w13_scale"][e],
-                                       host["w2"][e], host["w2_scale"][e], gate_first=bool(eng.cfg.gate_first))
+            yr, cq, cs = oracle.mlp_row(host["hidden_fp8"][t], xs, host["w13"][e], host["w13_scale"][e],
+                                        host["w2"][e], host["w2_scale"][e], gate_first=bool(eng.cfg.gate_first))
             assert np.allclose(a2s[r], cs, rtol=1e-5, atol=0), "re-quantisation scales differ"
             mism += int((a2[r] != cq).sum())
             tot += cq.size
+            # the slot's down-projection row (bf16 in the kernel, fp32 in the oracle), before the weighted combine
+            yg = yrows[int(r)]
+            y_bad += int((np.abs(yg - yr) > 1e-2 + 5e-2 * np.abs(yr)).sum())
+            y_tot += yr.size
         stats["a2_mismatch"] = mism / tot
         assert mism / tot <= 2e-3, f"{mism}/{tot} re-quantised codes differ"
+        stats["y_rows_bad"] = y_bad / y_tot
+        assert y_bad / y_tot <= 5e-3, f"{y_bad}/{y_tot} elements of the per-slot GEMM2 rows outside the tolerance"
     if own:
         eng.close()
     return stats
