@@ -70,7 +70,10 @@ int moe_fp8_destroy(moe_fp8_handle_t h);
 /* Bytes of device scratch needed for cfg.max_tokens tokens. */
 size_t moe_fp8_workspace_bytes(moe_fp8_handle_t h);
 /* Hands the library a caller-owned device buffer (1024-byte aligned) that must
- * stay valid until it is replaced or the handle destroyed. */
+ * stay valid until it is replaced or the handle destroyed.  The call zeroes two
+ * control words in it (synchronously, on the default stream); after that the
+ * contents belong to the library: a counter lives there between forwards, so
+ * the caller must not write into the buffer. */
 int moe_fp8_set_workspace(moe_fp8_handle_t h, void* dev_workspace, size_t bytes);
 
 /*

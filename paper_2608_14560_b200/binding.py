@@ -105,7 +105,7 @@ class MoeFp8:
 
     def __init__(self, hidden=7168, intermediate=2048, num_experts=256, num_local_experts=32, n_group=8,
                  topk_group=4, top_k=8, max_tokens=1024, hidden_scale_layout=0, gate_first=True,
-                 device="cuda:0"):
+                 device="cuda:0", poison_workspace=False):
         self.lib = load_library()
         self.cfg = Config(hidden, intermediate, num_experts, num_local_experts, n_group, topk_group, top_k,
                           max_tokens, hidden_scale_layout, int(gate_first))
@@ -116,6 +116,9 @@ class MoeFp8:
         self._check(self.lib.moe_fp8_create(C.byref(self.cfg), C.byref(self.handle)))
         self.workspace_bytes = int(self.lib.moe_fp8_workspace_bytes(self.handle))
         self.workspace = torch.empty(self.workspace_bytes + 1024, dtype=torch.uint8, device=self.device)
+        if poison_workspace:  # tests: scratch that is read before it is written shows up as NaN / -1
+            self.workspace.fill_(0xFF)
+            torch.cuda.synchronize(self.device)
         base = self.workspace.data_ptr()
         self._ws_ptr = (base + 1023) // 1024 * 1024
         self._check(self.lib.moe_fp8_set_workspace(self.handle, C.c_void_p(self._ws_ptr), self.workspace_bytes))

@@ -260,6 +260,9 @@ size_t moe_fp8_workspace_bytes(moe_fp8_handle_t h) { return h ? h->L.total : 0; 
 int moe_fp8_set_workspace(moe_fp8_handle_t h, void* ws, size_t bytes) {
     if (!h || !ws || (reinterpret_cast<uintptr_t>(ws) % WS_ALIGN) != 0) return MOE_FP8_ERR_BAD_ARG;
     if (bytes < h->L.total) return MOE_FP8_ERR_NO_WORKSPACE;
+    // the device status word and the ticket counter of route_permute_kernel start at zero
+    cudaError_t e = cudaMemset(static_cast<uint8_t*>(ws) + h->L.status, 0, 2 * sizeof(int));
+    if (e != cudaSuccess) return cuda_fail(h, e);
     h->ws = static_cast<uint8_t*>(ws);
     h->ws_bytes = bytes;
     if (!encode_2d(h, &h->tm_a1, h->ws + h->L.a1, h->L.row_cap, h->cfg.hidden, 1, 128, TILE_M,
@@ -326,8 +329,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     // next kernel cost the running GEMM about 6 %, so it is limited to the launch-latency-bound regime.
     const bool pdl = !h->stage_timing && T <= PDL_MAX_TOKENS;
 
-    cudaError_t e = cudaMemsetAsync(status, 0, 2 * sizeof(int), stream);  // status and ticket
-    if (e != cudaSuccess) return cuda_fail(h, e);
+    // No memset: the first kernel clears the status word, and the ticket counter returns to zero by itself.
     int ev_i = 0;
     auto mark = [&]() {
         if (h->stage_timing) cudaEventRecord(h->ev[ev_i++], stream);
@@ -358,7 +360,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         {  // stage 1: routing
             const int grid = min((T + 7) / 8, h->sm_count * 8);
             launch(route_topk_kernel, grid, 256, 0, stream, false, T, router_logits,
-                   static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w);
+                   static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w, status);
             ++launches;
             mark();
         }
@@ -432,7 +434,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         ++launches;
         mark();
     }
-    e = cudaGetLastError();
+    const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches = launches;
     h->stage_times_valid = h->stage_timing;

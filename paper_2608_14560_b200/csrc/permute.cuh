@@ -161,6 +161,7 @@ __global__ void __launch_bounds__(P_FUSED_THREADS) route_permute_small_kernel(
     __shared__ int s_cnt[P_MAX_LOCAL + 1];
     __shared__ int s_pad[P_MAX_LOCAL + 1];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) *status = DEV_OK;  // first kernel of a forward: clear the fault word
     for (int i = tid; i < E_loc * (P_TOKENS_PER_BLOCK / 32); i += blockDim.x) (&mask[0][0])[i] = 0u;
     {   // stage 1: one warp per token
         float bias_f[8];
@@ -247,7 +248,8 @@ __global__ void __launch_bounds__(P_FUSED_THREADS) route_permute_small_kernel(
 // Batches up to P_TAIL_MAX_TOKENS: routing in parallel blocks (one warp per token), then the block that
 // finishes last -- found with a ticket counter, nobody waits -- builds histogram, scan and placement for all
 // tokens on its own.  One launch instead of four; same arithmetic and outputs as route_topk_kernel +
-// count_kernel + scan_kernel + place_kernel.  `ticket` must be zero at launch; the last block leaves it zero.
+// count_kernel + scan_kernel + place_kernel.  `ticket` must be zero at launch; the last block leaves it zero
+// (moe_fp8_set_workspace zeroes it once, nothing else ever writes it).
 // Dynamic shared memory: E_loc * ceil(T/32) words of masks, then as many 16-bit prefix counts.
 constexpr int P_TAIL_MAX_TOKENS = 512;   // measured faster than the four kernels up to here, slower at 1024
 constexpr int P_TAIL_THREADS = 256;
@@ -265,6 +267,7 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
     __shared__ int s_pad[P_MAX_LOCAL + 1];
     __shared__ int s_last;
     const int tid = threadIdx.x, lane = tid & 31;
+    if (blockIdx.x == 0 && tid == 0) *status = DEV_OK;  // first kernel of a forward: clear the fault word
     {   // stage 1: one warp per token
         const int warps_per_block = blockDim.x >> 5;
         const int nwarps = gridDim.x * warps_per_block;

@@ -143,9 +143,11 @@ __device__ __forceinline__ void route_token(int t, int lane, const float* __rest
 
 __global__ void __launch_bounds__(256) route_topk_kernel(int T, const float* __restrict__ logits,
                                                          const __nv_bfloat16* __restrict__ bias, float scaling,
-                                                         int* __restrict__ topk_idx, float* __restrict__ topk_w) {
+                                                         int* __restrict__ topk_idx, float* __restrict__ topk_w,
+                                                         int* __restrict__ status) {
     pdl_launch_dependents();
     pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0) *status = DEV_OK;  // first kernel of a forward: clear the fault word
     const int lane = threadIdx.x & 31;
     const int warps_per_block = blockDim.x >> 5;
     const int warp0 = blockIdx.x * warps_per_block + (threadIdx.x >> 5);

@@ -51,9 +51,8 @@ def oracle_forward_parallel(host: dict, dims: syn.LayerDims, tokens, workers: in
 def make_engine(wl: syn.Workload, device, max_tokens=None, poison=True, **kw) -> MoeFp8:
     d = wl.dims
     eng = MoeFp8(d.hidden, d.intermediate, d.num_experts, d.num_local_experts, d.n_group, d.topk_group, d.top_k,
-                 max_tokens=max(wl.tokens, 1) if max_tokens is None else max_tokens, device=device, **kw)
-    if poison:
-        eng.workspace.fill_(0xFF)  # unwritten scratch reads as NaN (fp8, fp32, bf16) or -1 (int32)
+                 max_tokens=max(wl.tokens, 1) if max_tokens is None else max_tokens, device=device,
+                 poison_workspace=poison, **kw)  # unwritten scratch reads as NaN (fp8, fp32, bf16) or -1 (int32)
     return eng
 
 
