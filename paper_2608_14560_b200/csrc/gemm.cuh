@@ -31,6 +31,10 @@
 namespace moe {
 
 constexpr int G_STAGES = 4;
+// The two MMA issuer threads take the even and the odd K-blocks.  A thread must see EVERY phase of a barrier it
+// waits on (a parity wait cannot tell the wanted phase from the one two earlier), so a stage must always fall
+// to the same issuer: the stage count has to be even.
+static_assert(G_STAGES % 2 == 0, "an odd stage count lets an issuer thread skip phases of full[s]");
 constexpr int G_BLOCK_K = 128;                          // K bytes per stage = one scale block
 constexpr int G_TILE_N = 256;                           // output columns per tile
 constexpr int G_HALF_N = 128;                           // columns handled by one epilogue warpgroup
