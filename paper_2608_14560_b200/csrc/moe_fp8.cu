@@ -155,9 +155,6 @@ PermuteMeta meta_of(moe_fp8_handle_t h) {
 }
 
 constexpr int PDL_MAX_TOKENS = 2048;
-// One block routes one token per warp: measured faster than the four separate kernels up to 32 tokens only.
-constexpr int FUSED_ROUTE_MAX_TOKENS = 32;
-static_assert(FUSED_ROUTE_MAX_TOKENS <= P_TOKENS_PER_BLOCK, "the fused kernel handles one block of tokens");
 constexpr int NUM_STAGES = 8;
 const char* const STAGE_NAMES[NUM_STAGES] = {"route_topk", "count", "scan", "place", "gather_rows",
                                              "gemm1_swiglu_quant", "gemm2", "combine"};
@@ -337,16 +334,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     h->stage_times_valid = false;
     mark();
 
-    if (T <= FUSED_ROUTE_MAX_TOKENS) {  // stages 1-2 without the gather in one block (one warp per token)
-        launch(route_permute_small_kernel, 1, P_FUSED_THREADS, 0, stream, false, T, EL, local_expert_offset, row_cap,
-               router_logits, static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w, m,
-               status);
-        ++launches;
-        mark();
-        mark();
-        mark();
-        mark();
-    } else if (T <= P_TAIL_MAX_TOKENS) {  // routing in parallel blocks, the last one to finish does stage 2
+    if (T <= P_TAIL_MAX_TOKENS) {  // routing in parallel blocks, the last one to finish does stage 2
         const int grid = min((T + 7) / 8, h->sm_count * 8);
         launch(route_permute_kernel, grid, P_TAIL_THREADS, route_permute_smem_bytes(T, EL), stream, false, T, EL,
                local_expert_offset, row_cap, router_logits, static_cast<const __nv_bfloat16*>(routing_bias),

@@ -147,104 +147,6 @@ __global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) place_kernel(int T, int E_
     }
 }
 
-// Small batches (T <= P_TOKENS_PER_BLOCK): routing, histogram, scan and placement in ONE block, so the
-// launch-latency-bound regime pays for one kernel instead of four.  Same arithmetic and same outputs as
-// route_topk_kernel + count_kernel + scan_kernel + place_kernel.
-constexpr int P_FUSED_THREADS = 1024;
-__global__ void __launch_bounds__(P_FUSED_THREADS) route_permute_small_kernel(
-    int T, int E_loc, int off, int row_cap, const float* __restrict__ logits, const __nv_bfloat16* __restrict__ bias,
-    float scaling, int* __restrict__ topk_idx, float* __restrict__ topk_w, PermuteMeta m, int* __restrict__ status) {
-    pdl_launch_dependents();
-    pdl_wait();
-    __shared__ uint32_t mask[P_MAX_LOCAL][P_TOKENS_PER_BLOCK / 32];
-    __shared__ int s_idx[P_TOKENS_PER_BLOCK][8];
-    __shared__ int s_cnt[P_MAX_LOCAL + 1];
-    __shared__ int s_pad[P_MAX_LOCAL + 1];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) *status = DEV_OK;  // first kernel of a forward: clear the fault word
-    for (int i = tid; i < E_loc * (P_TOKENS_PER_BLOCK / 32); i += blockDim.x) (&mask[0][0])[i] = 0u;
-    {   // stage 1: one warp per token
-        float bias_f[8];
-        load_bias8(bias, lane, bias_f);
-        for (int t = warp; t < T; t += P_FUSED_THREADS / 32) {
-            int my_idx;
-            float my_w;
-            route_token(t, lane, logits, bias_f, scaling, my_idx, my_w);
-            if (lane < R_TOPK) {
-                topk_idx[t * R_TOPK + lane] = my_idx;
-                topk_w[t * R_TOPK + lane] = my_w;
-                s_idx[t][lane] = my_idx;
-            }
-        }
-    }
-    __syncthreads();
-    if (tid < T) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int e = s_idx[tid][j] - off;
-            if (e >= 0 && e < E_loc) atomicOr(&mask[e][tid >> 5], 1u << (tid & 31));
-        }
-    }
-    __syncthreads();
-    int total = 0;
-    if (tid < P_MAX_LOCAL) {
-        if (tid < E_loc) {
-#pragma unroll
-            for (int w = 0; w < P_TOKENS_PER_BLOCK / 32; ++w) total += __popc(mask[tid][w]);
-        }
-        s_cnt[tid] = total;
-        s_pad[tid] = (total + TILE_M - 1) / TILE_M * TILE_M;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int a = 0, p = 0;
-        for (int i = 0; i < E_loc; ++i) {
-            const int c = s_cnt[i], q = s_pad[i];
-            s_cnt[i] = a;
-            s_pad[i] = p;
-            a += c;
-            p += q;
-        }
-        s_cnt[E_loc] = a;
-        s_pad[E_loc] = p;
-        *m.num_m_tiles = p / TILE_M;
-        m.expert_offset[E_loc] = a;
-        m.padded_offset[E_loc] = p;
-    }
-    __syncthreads();
-    if (tid < E_loc) {
-        m.expert_count[tid] = total;
-        m.expert_offset[tid] = s_cnt[tid];
-        m.padded_offset[tid] = s_pad[tid];
-        const int t0 = s_pad[tid] / TILE_M;
-        for (int i = 0; i * TILE_M < total; ++i) {
-            m.tile_expert[t0 + i] = tid;
-            m.tile_rows[t0 + i] = min(TILE_M, total - i * TILE_M);
-        }
-    }
-    if (tid < T) {
-        const int word = tid >> 5, bit = tid & 31;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int e = s_idx[tid][j] - off;
-            int prow = -1;
-            if (e >= 0 && e < E_loc) {
-                int rank = __popc(mask[e][word] & ((1u << bit) - 1u));
-                for (int w = 0; w < word; ++w) rank += __popc(mask[e][w]);
-                prow = s_pad[e] + rank;
-                if (prow < 0 || prow >= row_cap) {
-                    atomicExch(status, DEV_BAD_ROW);
-                    prow = -1;
-                } else {
-                    m.row_to_slot[s_cnt[e] + rank] = tid * 8 + j;
-                    m.row_token[prow] = tid;
-                }
-            }
-            m.slot_to_row[tid * 8 + j] = prow;
-        }
-    }
-}
-
 // Batches up to P_TAIL_MAX_TOKENS: routing in parallel blocks (one warp per token), then the block that
 // finishes last -- found with a ticket counter, nobody waits -- builds histogram, scan and placement for all
 // tokens on its own.  One launch instead of four; same arithmetic and outputs as route_topk_kernel +
