@@ -117,6 +117,26 @@ def test_run_to_run_determinism_and_workspace_reuse(cuda_device):
     eng.close()
 
 
+def test_many_batch_sizes_back_to_back_on_one_handle(cuda_device):
+    # 600 forwards in random order over batch sizes on both sides of every launch-scheme boundary: the counters
+    # and scratch a forward leaves behind must never change the next one (bit-identical outputs, clean status)
+    sizes = [1, 8, 32, 33, 128, 129, 512, 513, 700, 2048, 2049]
+    inputs = {T: syn.make_inputs(_wl(T, seed=300 + T, skew=(T % 3 == 0)), cuda_device) for T in sizes}
+    eng = make_engine(_wl(max(sizes)), cuda_device)
+    want = {T: eng.forward(inputs[T]).clone() for T in sizes}
+    torch.cuda.synchronize()
+    assert eng.status() == 0
+    order = np.random.default_rng(5).choice(len(sizes), 600)
+    for i, k in enumerate(order):
+        T = sizes[k]
+        got = eng.forward(inputs[T])
+        if i % 20 == 19:
+            assert torch.equal(got.view(torch.int16), want[T].view(torch.int16)), f"forward {i}, T={T}"
+            assert eng.status() == 0
+    run_and_compare(_wl(129, seed=300 + 129, skew=True), cuda_device, inp=inputs[129], eng=eng)
+    eng.close()
+
+
 def test_host_entry_point_matches_device_entry_point(cuda_device):
     wl = _wl(260, seed=12)
     inp = syn.make_inputs(wl, cuda_device)
