@@ -381,7 +381,8 @@ def main():
                 continue
             w = syn.CONFIGS[i]
             st = args.steps if w.tokens <= 1024 else max(5, args.steps // 5)
-            r = run_cuda_config(w, device, st, max(3, args.warmup), peaks, peak_kind, want_e2e=False)
+            r = run_cuda_config(w, device, st, max(3, args.warmup), peaks, peak_kind, want_e2e=False,
+                                sampler_index=physical_gpu_index(local_rank))
             r.pop("total_ms")
             others.append(r)
 
