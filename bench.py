@@ -6,6 +6,9 @@ GEMM2, combine) over one batch of synthetic tokens.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config i] [--impl reference]
 
+The headline workload is the largest single-GPU configuration (all 256 experts
+local, T = 16384); the other four benchmark configurations and a sweep over
+token counts on the 32-local-expert layer are reported beside it at N = 1.
 N > 1 is launched under torch.distributed.run; every rank runs an independent
 replica of the layer on its own batch (no data-path collective, weak scaling).
 `--impl reference` times the CPU oracle (a deliberately plain program) on the
@@ -35,14 +38,21 @@ W13_BYTES_PER_EXPERT = 4096 * 7168 + 32 * 56 * 4
 W2_BYTES_PER_EXPERT = 7168 * 2048 + 56 * 16 * 4
 FP8_DATASHEET_TFLOPS = 4500.0
 HBM_DATASHEET_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of the headline
-# workload (profiles/launches_dsv3_T64_E32.md), mean over the two rotating activation sets.
-NCU_TRAFFIC_BYTES = {
-    ("dsv3_T64_E32", "gemm1_swiglu_quant"): (486.1e6 + 4.4e6 + 455.7e6 + 0.7e6) / 2,
-    ("dsv3_T64_E32", "gemm2"): (239.5e6 + 3.2e6 + 224.5e6 + 2.6e6) / 2,
+# Measured DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch divided by the algorithmic
+# bytes of the same launch, from the committed ncu captures (see profiles/): the weight-streaming regime was
+# captured on the T = 64 workload itself, the tensor-bound regime on a reduced case (32 local experts) whose
+# traffic is scaled to a full launch by the algorithmic bytes, since both grow with the experts and rows.
+NCU_TRAFFIC_RATIO = {
+    ("hbm", "gemm1_swiglu_quant"): 1.035, ("hbm", "gemm2"): 1.02,
+    ("tensor", "gemm1_swiglu_quant"): 1.14, ("tensor", "gemm2"): 1.10,
 }
 METRIC = "fused FP8 MoE forward throughput (tokens/s; TFLOPS and roofline fraction alongside)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+HEADLINE = 4
+# Token counts of the sweep over the three batch-size regimes of the paper's table of Fused MoE workload
+# groups (T = 1-16 / 32-80 / 901-14107), on the 32-local-expert layer; the paper quotes one latency per regime.
+SWEEP_TOKENS = (1, 2, 4, 7, 8, 16, 32, 54, 64, 80, 901, 4096, 14107)
+PAPER_MS = {7: 0.099, 54: 0.205, 14107: 1.229}
 
 
 def load_peaks():
@@ -138,7 +148,8 @@ def time_steps(eng, weights, acts, outs, flush, steps, stage=False):
     (untimed) precedes each step and the activation sets are rotated.  The flush
     writes one buffer larger than L2 and then reads a second one: the read pushes
     the dirty lines of the write out, so their write-back to HBM does not land
-    inside the timed region (it cost the first GEMM about 15 % of its bandwidth)."""
+    inside the timed region (it cost the first GEMM about 15 % of its bandwidth).
+    -> (per-step milliseconds, per-step stage times)."""
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     stage_ms = []
     for i in range(steps):
@@ -151,19 +162,44 @@ def time_steps(eng, weights, acts, outs, flush, steps, stage=False):
         if stage:
             stage_ms.append(eng.get_stage_times())
     torch.cuda.synchronize()
-    total = sum(s.elapsed_time(e) for s, e in ev)
-    return total, stage_ms
+    return [s.elapsed_time(e) for s, e in ev], stage_ms
+
+
+def time_warm(eng, weights, acts, outs, steps):
+    """Back-to-back forwards, no flush in between (activation sets still rotate): the warm figure."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(3):
+        eng.forward({**weights, **acts[i % len(acts)]}, out=outs[i % len(outs)])
+    e0.record()
+    for i in range(steps):
+        eng.forward({**weights, **acts[i % len(acts)]}, out=outs[i % len(outs)])
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def checksum64(t: torch.Tensor) -> int:
+    """Wrap-around 64-bit sum over the tensor's bytes taken as little-endian int64 words."""
+    b = t.contiguous().view(torch.uint8).flatten()
+    n8 = b.numel() // 8 * 8
+    total = int(b[:n8].view(torch.int64).sum().item()) if n8 else 0
+    if n8 < b.numel():
+        total += int(b[n8:].to(torch.int64).sum().item())
+    return total & 0xFFFFFFFFFFFFFFFF
 
 
 def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, cpu_baseline=False,
-                    sampler_index=None):
+                    sampler_index=None, inp=None, checksums=False):
+    """One workload on the CUDA path.  `inp` may carry prebuilt inputs of the same layer with at least
+    wl.tokens tokens (the sweep re-uses one set of weights)."""
     from paper_2608_14560_b200 import MoeFp8
     d = wl.dims
     T = wl.tokens
-    inp = syn.make_inputs(wl, device)
+    if inp is None:
+        inp = syn.make_inputs(wl, device)
     weights = {k: inp[k] for k in ("routing_bias", "w13", "w13_scale", "w2", "w2_scale", "local_expert_offset",
                                    "scaling_factor")}
-    acts = [{k: inp[k] for k in ("hidden_fp8", "hidden_scale", "router_logits")},
+    acts = [{k: inp[k][:T] for k in ("hidden_fp8", "hidden_scale", "router_logits")},
             syn.make_activations(wl, wl.seed + 1000, device)]
     outs = [torch.empty(T, d.hidden, dtype=torch.bfloat16, device=device) for _ in range(2)]
     flush = [torch.zeros(256 << 20, dtype=torch.uint8, device=device) for _ in range(2)]
@@ -186,13 +222,15 @@ def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, 
     if world > 1:
         torch.distributed.barrier()
     torch.cuda.synchronize()
-    total_ms, _ = time_steps(eng, weights, acts, outs, flush, steps)
+    step_ms, _ = time_steps(eng, weights, acts, outs, flush, steps)
     torch.cuda.synchronize()
     if world > 1:
         torch.distributed.barrier()
+    total_ms = sum(step_ms)
     launches = eng.last_launch_count() * steps
     status = eng.status()
     assert status == 0, f"device status {status} after the timed region"
+    warm_ms = time_warm(eng, weights, acts, outs, steps)
 
     # per-kernel device times over the same kind of region (events around every launch)
     eng.set_stage_timing(True)
@@ -203,19 +241,24 @@ def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, 
         sampler.stop_flag = True
         sampler.join()
     stage_avg = {k: float(np.mean([s[k] for s in stage_ms])) for k in stage_ms[0]}
+    stage_med = {k: float(np.median([s[k] for s in stage_ms])) for k in stage_ms[0]}
 
     ms = total_ms / steps
+    ms_med = float(statistics.median(step_ms))
     flops = FLOPS_PER_SLOT * S * (d.hidden * d.intermediate) / (7168 * 2048)
     t_flop = flops / (FP8_DATASHEET_TFLOPS * 1e12)
     t_hbm = BYTES_PER_EXPERT * A / (HBM_DATASHEET_GBS * 1e9)
     bound = "tensor" if t_flop > t_hbm else "hbm"
     res = {
-        "workload": wl.name, "tokens": T, "local_slots": S, "active_experts": A, "ms_per_step": ms,
+        "workload": wl.name, "tokens": T, "local_slots": S, "active_experts": A, "steps": steps,
+        "ms_per_step": ms, "ms_per_step_median": ms_med, "ms_per_step_min": min(step_ms),
+        "ms_per_step_warm": warm_ms,
         "tokens_per_s": T / (ms * 1e-3), "tflops": flops / (ms * 1e-3) / 1e12,
         "weight_gbs": BYTES_PER_EXPERT * A / (ms * 1e-3) / 1e9,
         "roofline_bound": bound, "roofline_frac_of_datasheet": max(t_flop, t_hbm) / (ms * 1e-3),
-        "stage_ms": stage_avg, "launches_per_step": eng.last_launch_count(), "total_ms": total_ms,
-        "gpu_launches": launches,
+        "roofline_frac_of_datasheet_median": max(t_flop, t_hbm) / (ms_med * 1e-3),
+        "stage_ms": stage_avg, "stage_ms_median": stage_med, "launches_per_step": eng.last_launch_count(),
+        "total_ms": total_ms, "gpu_launches": launches,
     }
     # roofline of the dominant kernel, against the measured peaks of this machine
     dom = max(stage_avg, key=stage_avg.get)
@@ -230,16 +273,28 @@ def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, 
         ach = kern_flops / dom_s / 1e12
         res["roofline"] = {"bound": "tensor", "kernel": dom, "achieved": ach, "peak": fp8_peak, "unit": "TFLOP/s",
                            "frac": ach / fp8_peak, "traffic": None,
-                           "peak_source": f"2 x {peak_kind} bf16 cuBLAS peak (fp8:bf16 nominal ratio 2)"}
+                           "frac_of_datasheet": ach / FP8_DATASHEET_TFLOPS,
+                           "peak_source": f"2 x {peak_kind} bf16 cuBLAS peak (fp8:bf16 nominal ratio 2), "
+                                          + ("sustained" if ms * steps > 500 else "burst")}
     else:
         ach = kern_bytes / dom_s / 1e9
         res["roofline"] = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                           "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": f"{peak_kind} copy bandwidth"}
-    res["roofline"]["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name, dom))
-    res["roofline"]["algorithmic_per_launch"] = kern_flops if res["roofline"]["bound"] == "tensor" else kern_bytes
+                           "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                           "frac_of_datasheet": ach / HBM_DATASHEET_GBS, "peak_source": f"{peak_kind} copy bandwidth"}
+    ratio = NCU_TRAFFIC_RATIO.get((res["roofline"]["bound"], dom))
+    res["roofline"]["traffic"] = None if ratio is None else ratio * kern_bytes
+    res["roofline"]["traffic_source"] = ("ncu capture of this kernel on a smaller case of the same regime, scaled "
+                                         "to this launch by its algorithmic bytes")
+    res["roofline"]["algorithmic_bytes_per_launch"] = kern_bytes
+    res["roofline"]["algorithmic_flops_per_launch"] = kern_flops
     res["roofline"]["kernel_ms"] = stage_avg[dom]
     if sampler:
         res["clocks"] = sampler.result()
+        mhz = res["clocks"]["sm_mhz"]
+        if mhz:  # time x clock: separates fewer cycles from a higher clock under the power cap
+            res["mcycles_per_step"] = ms_med * mhz * 1e-3
+    if checksums:
+        res["input_checksums"] = {k: f"{checksum64(v):016x}" for k, v in inp.items() if torch.is_tensor(v)}
 
     if want_e2e:
         host_acts = [{k: v.cpu().pin_memory() for k, v in a.items()} for a in acts]
@@ -247,19 +302,21 @@ def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, 
         for i in range(3):
             eng.forward_host(host_acts[i % 2], weights, host_out)
         torch.cuda.synchronize()
+        e2e_steps = min(steps, 50)
         t0 = time.perf_counter()
-        for i in range(steps):
+        for i in range(e2e_steps):
             eng.forward_host(host_acts[i % 2], weights, host_out)
-        e2e_s = (time.perf_counter() - t0) / steps
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
         h2d = sum(v.numel() * v.element_size() for v in host_acts[0].values())
-        res["e2e"] = {"value": T / e2e_s, "unit": "tokens/s", "ms_per_step": e2e_s * 1e3,
+        res["e2e"] = {"value": T / e2e_s, "unit": "tokens/s", "ms_per_step": e2e_s * 1e3, "steps": e2e_steps,
                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": host_out.numel() * 2,
                       "checksum": float(host_out.float().abs().sum())}
+        del host_acts, host_out
 
     if cpu_baseline:
-        res["cpu_baseline"] = oracle_baseline(wl, syn.to_host(inp))
+        res["cpu_baseline"] = oracle_baseline(wl, syn.to_host(inp), S / T)
     eng.close()
-    del eng, inp, weights, acts, outs
+    del eng, weights, acts, outs
     torch.cuda.empty_cache()
     return res
 
@@ -277,11 +334,18 @@ def oracle_sample_tokens(wl, budget_slots=400):
     return np.arange(n, dtype=np.int32)
 
 
-def oracle_baseline(wl, host, min_seconds=10.0):
-    """The oracle as it stands, one thread, on a bounded token sample, repeated until ~10 s of CPU work."""
+def oracle_baseline(wl, host, slots_per_token, min_seconds=10.0):
+    """The oracle as it stands on a bounded token sample: one thread, repeated until ~10 s of CPU work, the
+    time per (token, expert) slot extrapolated to the whole workload by its slot count; then the same sample
+    once more with one unmodified single-thread oracle call per core (threads, the C call releases the GIL)."""
     import oracle
+    from concurrent.futures import ThreadPoolExecutor
     d = wl.dims
     tokens = oracle_sample_tokens(wl)
+    idx, _ = oracle.route(host["router_logits"], host["routing_bias"], d.n_group, d.topk_group, d.top_k,
+                          float(host["scaling_factor"]))
+    off = int(host["local_expert_offset"])
+    sample_slots = int(((idx[tokens] >= off) & (idx[tokens] < off + d.num_local_experts)).sum())
     t0 = time.perf_counter()
     reps = 0
     while True:
@@ -291,9 +355,20 @@ def oracle_baseline(wl, host, min_seconds=10.0):
             break
     total = time.perf_counter() - t0
     dt = total / reps
-    return {"value": len(tokens) / dt, "unit": "tokens/s", "cores": 1, "kind": "oracle",
-            "sample": f"first {len(tokens)} of {wl.tokens} tokens of {wl.name} (routing on all tokens), "
-                      f"single thread, {reps} pass(es), {total:.1f} s in total", "host_cores": os.cpu_count()}
+    s_per_slot = dt / max(sample_slots, 1)
+    cores = os.cpu_count() or 1
+    shards = [x for x in np.array_split(tokens, min(cores, len(tokens))) if x.size]
+    t1 = time.perf_counter()
+    with ThreadPoolExecutor(len(shards)) as ex:
+        list(ex.map(lambda x: oracle.forward(host, d.n_group, d.topk_group, d.top_k, tokens=x), shards))
+    dt_all = time.perf_counter() - t1
+    return {"value": 1.0 / (s_per_slot * max(slots_per_token, 1e-9)), "unit": "tokens/s", "cores": 1, "kind": "oracle",
+            "sample": f"first {len(tokens)} of {wl.tokens} tokens of {wl.name} ({sample_slots} local slots; routing on "
+                      f"all tokens), single thread, {reps} pass(es), {total:.1f} s in total; extrapolated to the "
+                      f"workload by slot count ({slots_per_token:.3f} local slots per token)",
+            "seconds_per_slot": s_per_slot, "host_cores": cores,
+            "all_cores": {"value": len(tokens) / dt_all, "unit": "tokens/s", "cores": len(shards),
+                          "sample": "the same sample split over one single-thread oracle call per core, one pass"}}
 
 
 def run_reference(args, wl):
@@ -330,22 +405,27 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=1, help="index into the five benchmark workloads (headline)")
+    ap.add_argument("--config", type=int, default=HEADLINE,
+                    help="index into the five benchmark workloads (headline; default: the largest single-GPU one)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--others", default="0,2,3,4", help="extra workloads reported under 'workloads' at N=1 ('' = none)")
+    ap.add_argument("--others", default="0,1,2,3", help="extra workloads reported under 'workloads' at N=1 ('' = none)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override T of the chosen workload (profiling runs)")
-    ap.add_argument("--paper-points", default="7,54,14107",
-                    help="token counts the paper quotes a latency for (its table of workload regimes: short / median / long); "
-                         "timed on the 32-local-expert layer and reported under 'paper_points' ('' = none)")
+    ap.add_argument("--local-experts", type=int, default=0,
+                    help="override the number of local experts of the chosen workload (reduced profiling cases)")
+    ap.add_argument("--sweep", default=",".join(str(t) for t in SWEEP_TOKENS),
+                    help="token counts timed on the 32-local-expert layer and reported under 'sweep' at N=1 ('' = none)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
     wl = syn.CONFIGS[args.config]
-    if args.tokens > 0:
-        wl = syn.Workload(f"{wl.name}_T{args.tokens}", args.tokens, wl.dims, wl.seed, wl.local_expert_offset,
+    if args.tokens > 0 or args.local_experts > 0:
+        import dataclasses
+        dims = dataclasses.replace(wl.dims, num_local_experts=args.local_experts) if args.local_experts > 0 else wl.dims
+        tk = args.tokens if args.tokens > 0 else wl.tokens
+        wl = syn.Workload(f"{wl.name}_T{tk}_E{dims.num_local_experts}", tk, dims, wl.seed, wl.local_expert_offset,
                           wl.scaling_factor, wl.skew)
 
     if args.impl == "reference":
@@ -361,12 +441,13 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
     peaks, peak_kind = load_peaks()
+    steps = max(args.steps, 1)
 
     my_wl = syn.Workload(wl.name, wl.tokens, wl.dims, wl.seed + 7919 * rank, wl.local_expert_offset,
                          wl.scaling_factor, wl.skew)
-    res = run_cuda_config(my_wl, device, args.steps, args.warmup, peaks, peak_kind, want_e2e=not args.no_e2e,
+    res = run_cuda_config(my_wl, device, steps, args.warmup, peaks, peak_kind, want_e2e=not args.no_e2e,
                           cpu_baseline=(rank == 0 and world == 1 and not args.no_cpu_baseline),
-                          sampler_index=physical_gpu_index(local_rank))
+                          sampler_index=physical_gpu_index(local_rank), checksums=True)
     total_ms = max_over_ranks(res["total_ms"], world, device)
     if args.no_e2e:
         res["e2e"] = {"ms_per_step": float("nan"), "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
@@ -374,39 +455,48 @@ def main():
     tokens_all = sum_over_ranks(float(my_wl.tokens), world, device)
     launches = sum_over_ranks(float(res["gpu_launches"]), world, device)
 
+    side_steps = max(20, min(steps, 100))  # every side workload gets at least 20 timed steps
     others = []
     if world == 1 and args.others:
         for i in [int(x) for x in args.others.split(",") if x != ""]:
             if i == args.config:
                 continue
-            w = syn.CONFIGS[i]
-            st = args.steps if w.tokens <= 1024 else max(5, args.steps // 5)
-            r = run_cuda_config(w, device, st, max(3, args.warmup), peaks, peak_kind, want_e2e=False,
-                                sampler_index=physical_gpu_index(local_rank))
+            r = run_cuda_config(syn.CONFIGS[i], device, side_steps, max(3, args.warmup), peaks, peak_kind,
+                                want_e2e=False, sampler_index=physical_gpu_index(local_rank))
             r.pop("total_ms")
             others.append(r)
 
-    # The paper's three quoted latencies (B200, 32 local experts of 256, contest workloads whose routing is not
-    # published): the same token counts on the synthetic layer of workload 1, as context.
-    paper_ms = {7: 0.099, 54: 0.205, 14107: 1.229}
-    points = []
-    if world == 1 and args.paper_points:
+    # Sweep over token counts on the 32-local-expert layer (one set of weights, drawn once for the largest T),
+    # with the paper's quoted latency beside the three counts it names (B200, its contest workloads, whose
+    # routing is not published: context only).
+    sweep = []
+    if world == 1 and args.sweep:
+        ts = sorted(int(x) for x in args.sweep.split(",") if x != "")
         base = syn.CONFIGS[1]
-        for t in [int(x) for x in args.paper_points.split(",") if x != ""]:
+        big = syn.Workload(f"dsv3_T{ts[-1]}_E32", ts[-1], base.dims, base.seed, base.local_expert_offset,
+                           base.scaling_factor, base.skew)
+        inp = syn.make_inputs(big, device)
+        for t in ts:
             w = syn.Workload(f"dsv3_T{t}_E32", t, base.dims, base.seed, base.local_expert_offset,
                              base.scaling_factor, base.skew)
-            st = args.steps if t <= 1024 else max(5, args.steps // 5)
-            r = run_cuda_config(w, device, st, max(3, args.warmup), peaks, peak_kind, want_e2e=False)
-            points.append({"tokens": t, "ms_per_step": r["ms_per_step"], "paper_ms": paper_ms.get(t),
-                           "local_slots": r["local_slots"], "active_experts": r["active_experts"],
-                           "tflops": r["tflops"], "weight_gbs": r["weight_gbs"]})
+            r = run_cuda_config(w, device, side_steps, max(3, args.warmup), peaks, peak_kind, want_e2e=False, inp=inp)
+            sweep.append({"tokens": t, "ms_per_step": r["ms_per_step"], "ms_per_step_median": r["ms_per_step_median"],
+                          "ms_per_step_warm": r["ms_per_step_warm"], "paper_ms": PAPER_MS.get(t),
+                          "local_slots": r["local_slots"], "active_experts": r["active_experts"],
+                          "tflops": r["tflops"], "weight_gbs": r["weight_gbs"],
+                          "roofline_bound": r["roofline_bound"],
+                          "roofline_frac_of_datasheet": r["roofline_frac_of_datasheet"],
+                          "launches_per_step": r["launches_per_step"]})
+        del inp
+        torch.cuda.empty_cache()
 
     if rank == 0:
-        ms = total_ms / args.steps
+        ms = total_ms / steps
         line = {
             "metric": METRIC,
-            "value": tokens_all / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "value": tokens_all / (ms * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms, "ms_per_step_median": res["ms_per_step_median"],
+            "ms_per_step_warm": res["ms_per_step_warm"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "fp8_e4m3 x fp8_e4m3 -> f32", "data": "synthetic",
             "config": {"workload": wl.name, "tokens_per_gpu": wl.tokens, "hidden": wl.dims.hidden,
                        "intermediate": wl.dims.intermediate, "local_experts": wl.dims.num_local_experts,
@@ -416,14 +506,16 @@ def main():
                        "stands_in_for": "FlashInfer-Bench Fused-MoE contest workloads (DeepSeek-V3 shapes)"},
             "tflops": res["tflops"] * world, "weight_gbs_per_gpu": res["weight_gbs"],
             "roofline_frac_of_datasheet": {"bound": res["roofline_bound"], "frac": res["roofline_frac_of_datasheet"],
+                                           "frac_median_step": res["roofline_frac_of_datasheet_median"],
                                            "fp8_tflops": FP8_DATASHEET_TFLOPS, "hbm_gbs": HBM_DATASHEET_GBS},
-            "roofline": res["roofline"], "stage_ms": res["stage_ms"],
+            "roofline": res["roofline"], "stage_ms": res["stage_ms"], "stage_ms_median": res["stage_ms_median"],
             "e2e": {"value": tokens_all / (e2e_ms * 1e-3), "unit": "tokens/s",
                     "h2d_bytes_per_step": res["e2e"]["h2d_bytes_per_step"],
                     "d2h_bytes_per_step": res["e2e"]["d2h_bytes_per_step"], "ms_per_step": e2e_ms},
             "gpu_launches": int(launches), "clocks": res.get("clocks"),
-            "cpu_baseline": res.get("cpu_baseline"), "peaks": peak_kind, "workloads": others,
-            "paper_points": points,
+            "mcycles_per_step": res.get("mcycles_per_step"),
+            "cpu_baseline": res.get("cpu_baseline"), "input_checksums": res.get("input_checksums"),
+            "peaks": peak_kind, "workloads": others, "sweep": sweep,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -71,7 +71,7 @@ int moe_fp8_destroy(moe_fp8_handle_t h);
 size_t moe_fp8_workspace_bytes(moe_fp8_handle_t h);
 /* Hands the library a caller-owned device buffer (1024-byte aligned) that must
  * stay valid until it is replaced or the handle destroyed.  The call zeroes two
- * control words in it (synchronously, on the default stream); after that the
+ * control words in it and waits for the device (cudaDeviceSynchronize); after that the
  * contents belong to the library: a counter lives there between forwards, so
  * the caller must not write into the buffer. */
 int moe_fp8_set_workspace(moe_fp8_handle_t h, void* dev_workspace, size_t bytes);
@@ -128,6 +128,22 @@ int moe_fp8_forward_host(moe_fp8_handle_t h, int T, const void* host_hidden_fp8,
 int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w, int* expert_count,
                          int* expert_offset, int* row_to_slot, void* a2_fp8, float* a2_scale, void* y_rows,
                          int* status_word, void* stream);
+
+/*
+ * Test hook for the failure path of the bounded device waits (every wait on an mbarrier inside the GEMM
+ * kernels gives up after a limit, records a fault code in the status word and lets the kernel return with
+ * its tensor memory released).  skip_iteration >= 0: in the next forwards the copy producer of every CTA
+ * of the GEMM1 kernel stops before its skip_iteration-th pipeline stage, so the consumers wait for a stage
+ * that nothing fills; wait_clocks > 0 shortens the limit of every wait to that many SM clocks (0 restores
+ * the default of about a second).  skip_iteration < 0 switches the hook off.  Nothing traps: the forward
+ * returns normally, its output is garbage and the status word holds a time-out code (1..5).
+ */
+int moe_fp8_debug_set_fault(moe_fp8_handle_t h, int skip_iteration, long long wait_clocks);
+
+/* Test hook: y[i] = the routing stage's sigmoid of x[i] (stage 1 of the Fused MoE description; the indices
+ * it selects are compared bit for bit, so its arithmetic is fixed operation by operation).  Device
+ * pointers, fp32 [n]; enqueued on `stream`. */
+int moe_fp8_debug_sigmoid(int n, const float* x, float* y, void* stream);
 
 /*
  * Measurement hook (the paper profiles each kernel of one MoE iteration, Appendix

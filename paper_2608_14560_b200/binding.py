@@ -17,7 +17,8 @@ EXPORTS = (
     "moe_fp8_create", "moe_fp8_destroy", "moe_fp8_workspace_bytes", "moe_fp8_set_workspace", "moe_fp8_forward",
     "moe_fp8_forward_host", "moe_fp8_debug_export", "moe_fp8_last_cuda_error", "moe_fp8_last_launch_count",
     "moe_fp8_strerror", "moe_fp8_set_stage_timing", "moe_fp8_num_stages", "moe_fp8_stage_name",
-    "moe_fp8_get_stage_times", "moe_fp8_expert_histogram_static",
+    "moe_fp8_get_stage_times", "moe_fp8_expert_histogram_static", "moe_fp8_debug_set_fault",
+    "moe_fp8_debug_sigmoid",
 )
 
 
@@ -74,6 +75,10 @@ def load_library() -> C.CDLL:
         lib.moe_fp8_get_stage_times.restype = C.c_int
         lib.moe_fp8_expert_histogram_static.argtypes = [C.c_int, ip, C.c_int, C.c_int, ip, ip, vp]
         lib.moe_fp8_expert_histogram_static.restype = C.c_int
+        lib.moe_fp8_debug_set_fault.argtypes = [vp, C.c_int, C.c_longlong]
+        lib.moe_fp8_debug_set_fault.restype = C.c_int
+        lib.moe_fp8_debug_sigmoid.argtypes = [C.c_int, fp, fp, vp]
+        lib.moe_fp8_debug_sigmoid.restype = C.c_int
         lib.moe_fp8_strerror.argtypes = [C.c_int]
         lib.moe_fp8_strerror.restype = C.c_char_p
         _lib = lib
@@ -94,10 +99,30 @@ def expert_histogram_static(topk_idx: torch.Tensor, local_expert_offset: int, nu
     workspace or allocation (for callers that may not allocate: graph capture, serving loops, plug-ins
     without a memory pool).  The caller passes the preallocated int32 outputs; returns the C return code."""
     lib = load_library()
+    for name, t, shape in (("topk_idx", topk_idx, None), ("expert_count", expert_count, (num_local_experts,)),
+                           ("expert_offset", expert_offset, (num_local_experts + 1,))):
+        if t.dtype != torch.int32 or not t.is_contiguous() or t.device != topk_idx.device or not t.is_cuda:
+            raise TypeError(f"{name} must be a contiguous int32 CUDA tensor on the device of topk_idx")
+        if shape is not None and tuple(t.shape) != shape:
+            raise ValueError(f"{name} must have shape {shape}")
+    if topk_idx.dim() != 2 or topk_idx.shape[1] != 8:
+        raise ValueError("topk_idx must have shape [T, 8]")
     s = torch.cuda.current_stream(topk_idx.device) if stream is None else stream
     return int(lib.moe_fp8_expert_histogram_static(
         int(topk_idx.shape[0]), _ptr(topk_idx), int(local_expert_offset), int(num_local_experts),
         _ptr(expert_count), _ptr(expert_offset), C.c_void_p(s.cuda_stream)))
+
+
+def debug_sigmoid(x: torch.Tensor, stream=None) -> torch.Tensor:
+    """moe_fp8_debug_sigmoid: the routing stage's sigmoid on a contiguous fp32 CUDA tensor."""
+    if x.dtype != torch.float32 or not x.is_contiguous() or not x.is_cuda:
+        raise TypeError("x must be a contiguous fp32 CUDA tensor")
+    y = torch.empty_like(x)
+    s = torch.cuda.current_stream(x.device) if stream is None else stream
+    rc = int(load_library().moe_fp8_debug_sigmoid(x.numel(), _ptr(x), _ptr(y), C.c_void_p(s.cuda_stream)))
+    if rc != OK:
+        raise MoeFp8Error(rc, load_library().moe_fp8_strerror(rc).decode())
+    return y
 
 
 class MoeFp8:
@@ -167,6 +192,10 @@ class MoeFp8:
             int(weights["local_expert_offset"]), float(weights["scaling_factor"]), _ptr(host_out),
             self._stream(stream)))
         return host_out
+
+    def debug_set_fault(self, skip_iteration: int = -1, wait_clocks: int = 0):
+        """moe_fp8_debug_set_fault (test hook of the bounded-wait failure path)."""
+        self._check(self.lib.moe_fp8_debug_set_fault(self.handle, int(skip_iteration), int(wait_clocks)))
 
     def set_stage_timing(self, enable: bool):
         self._check(self.lib.moe_fp8_set_stage_timing(self.handle, int(enable)))

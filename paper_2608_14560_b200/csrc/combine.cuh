@@ -13,9 +13,8 @@ namespace moe {
 
 // y is the tile-blocked bf16 output of GEMM2 (see y_block_offset); each thread owns 16 columns
 // (one 32-byte group) of one token.
-__global__ void __launch_bounds__(256) combine_kernel(int T, int H, const int* __restrict__ slot_to_row,
-                                                      const float* __restrict__ topk_w,
-                                                      const uint8_t* __restrict__ y,
+__global__ void __launch_bounds__(256) combine_kernel(int T, int H, const int* slot_to_row, const float* topk_w,
+                                                      const uint8_t* y,
                                                       __nv_bfloat16* __restrict__ out) {
     pdl_launch_dependents();
     pdl_wait();
@@ -25,8 +24,8 @@ __global__ void __launch_bounds__(256) combine_kernel(int T, int H, const int* _
         float w[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            rows[j] = __ldg(slot_to_row + t * 8 + j);
-            w[j] = __ldg(topk_w + t * 8 + j);
+            rows[j] = __ldcg(slot_to_row + t * 8 + j);  // written by the kernels before this one: coherent loads
+            w[j] = __ldcg(topk_w + t * 8 + j);
         }
         for (int c = threadIdx.x; c < groups; c += blockDim.x) {
             float acc[16];
@@ -36,7 +35,7 @@ __global__ void __launch_bounds__(256) combine_kernel(int T, int H, const int* _
             for (int j = 0; j < 8; ++j) {
                 if (rows[j] < 0) continue;
                 uint32_t u[8];
-                ld_global_nc_v8(y + y_block_offset(rows[j], c, n_tiles), u);
+                ld_global_v8(y + y_block_offset(rows[j], c, n_tiles), u);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     acc[2 * i] = fmaf(w[j], __uint_as_float(u[i] << 16), acc[2 * i]);

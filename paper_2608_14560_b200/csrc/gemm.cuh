@@ -7,7 +7,8 @@
 //   warp 0      TMA producer.  Per K-block (128 K-bytes = one scale block): the A
 //               tile (128 rows), the B tile (256 weight rows) and the 128
 //               activation scales of the block, into a 4-stage ring (128-byte
-//               swizzle) / an 8-slot scale ring, completion on mbarriers.
+//               swizzle) / an 8-slot scale ring (its own mbarrier per slot, so the
+//               epilogue can fetch a scale before the MMAs that use the block end).
 //   warps 1,2   MMA issuers (even / odd K-blocks).  Four tcgen05.mma (M128 N256 K32, e4m3 -> fp32) per
 //               K-block into one of two 256-column TMEM buffers, then ONE
 //               tcgen05.commit: the same mbarrier tells the producer that the stage
@@ -71,11 +72,14 @@ struct GemmArgs {
     float* out_scale_t;       // GEMM1: [I/128, row_cap]
     __nv_bfloat16* out_bf16;  // GEMM2: tile-blocked rows, see y_block_offset()
     int* status;
+    long long wait_limit;     // clocks a bounded wait may spin (WAIT_LIMIT_CLOCKS outside of tests)
+    int fault_skip_it;        // test hook: the producer stops before this pipeline iteration (-1: never)
 };
 
 struct GemmCtrl {
     uint64_t full[G_STAGES];   // stage filled (TMA transaction bytes)
     uint64_t done[G_STAGES];   // the MMAs that read the stage have finished: stage free AND accumulator ready
+    uint64_t scale_full[G_SCALE_RING];  // activation scales of a K-block have landed
     uint64_t tmem_empty[G_ACC_BUFS];
     uint64_t amax_bar[2];
     uint64_t drain_bar[2];
@@ -111,6 +115,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(smem_u32(&ctrl->full[s]), 1);
             mbar_init(smem_u32(&ctrl->done[s]), 1);
         }
+        for (int s = 0; s < G_SCALE_RING; ++s) mbar_init(smem_u32(&ctrl->scale_full[s]), 1);
         for (int b = 0; b < G_ACC_BUFS; ++b) {
             mbar_init(smem_u32(&ctrl->tmem_empty[b]), G_EPI_WARPS);
         }
@@ -138,8 +143,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     pdl_launch_dependents();
     pdl_wait();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_slot);
-    const int num_tiles = __ldg(g.num_m_tiles) * g.n_tiles;
+    // (the tables come from the kernels before this one, which may still be resident: coherent loads)
+    const int num_tiles = __ldcg(g.num_m_tiles) * g.n_tiles;
     const int num_kb = g.num_kb;
+    const long long limit = g.wait_limit;
 
     if (warp < 4) {
         reg_dealloc<40>();
@@ -149,11 +156,15 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
-                const int wrow = __ldg(g.tile_expert + m_tile) * g.w_rows_per_expert;
+                const int wrow = __ldcg(g.tile_expert + m_tile) * g.w_rows_per_expert;
                 const float* a_sc = g.a_scale_t + static_cast<size_t>(m_tile) * TILE_M;
                 for (int kb = 0; kb < num_kb; ++kb, ++it) {
                     const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1;
-                    if (!mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, abort_flag)) {
+                    if (static_cast<int>(it) == g.fault_skip_it) {  // test hook: this stage is never filled
+                        ok = false;
+                        break;
+                    }
+                    if (!mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, abort_flag, limit)) {
                         raise(ctrl, g.status, DEV_TIMEOUT_PRODUCER);
                         ok = false;
                         break;
@@ -161,7 +172,13 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t bar = smem_u32(&ctrl->full[s]);
                     const uint32_t a_dst = smem_base + s * G_STAGE_BYTES, b_dst = a_dst + G_A_BYTES;
                     const int k0 = kb * G_BLOCK_K;
-                    mbar_expect_tx(bar, G_STAGE_BYTES + G_SCALE_BYTES);
+                    // The scale slot is free: 8 slots exceed the 4 stages + 2 accumulators the producer can
+                    // be ahead of the epilogue.
+                    const uint32_t sbar = smem_u32(&ctrl->scale_full[it % G_SCALE_RING]);
+                    mbar_expect_tx(sbar, G_SCALE_BYTES);
+                    bulk_load_1d(smem_u32(scale_ring + (it % G_SCALE_RING) * TILE_M),
+                                 a_sc + static_cast<size_t>(kb) * g.row_cap, G_SCALE_BYTES, sbar);
+                    mbar_expect_tx(bar, G_STAGE_BYTES);
                     tma_load_2d(a_dst, &tmA, k0, m_tile * TILE_M, bar);
                     if (MODE == 1) {
                         const int gr = wrow + g.gate_row0 + n * 128, ur = wrow + g.up_row0 + n * 128;
@@ -174,16 +191,21 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         tma_load_2d(b_dst, &tmB, k0, br, bar);
                         tma_load_2d(b_dst + G_B_BYTES / 2, &tmB, k0, br + 128, bar);
                     }
-                    bulk_load_1d(smem_u32(scale_ring + (it % G_SCALE_RING) * TILE_M),
-                                 a_sc + static_cast<size_t>(kb) * g.row_cap, G_SCALE_BYTES, bar);
                 }
             }
-            if (!ok || *abort_flag) {
-                // wait (bounded) until the copies still in flight have landed
-                const uint32_t n_back = it < G_STAGES ? it : G_STAGES;
+            {
+                // Before this thread may reach the end of the kernel every copy it issued has to have landed
+                // (bounded wait).  On the regular path the MMA issuers have consumed all of them long ago and
+                // these waits fall through; after an abort raised by any role they are what keeps the
+                // copy engine from writing into shared memory of a CTA that has exited.
                 int zero = 0;
+                const uint32_t n_back = it < G_STAGES ? it : G_STAGES;
                 for (uint32_t j = it - n_back; j < it; ++j)
-                    if (!mbar_wait(smem_u32(&ctrl->full[j % G_STAGES]), (j / G_STAGES) & 1, &zero))
+                    if (!mbar_wait(smem_u32(&ctrl->full[j % G_STAGES]), (j / G_STAGES) & 1, &zero, limit))
+                        atomicCAS(g.status, DEV_OK, DEV_TIMEOUT_DRAIN);
+                const uint32_t s_back = it < G_SCALE_RING ? it : G_SCALE_RING;
+                for (uint32_t j = it - s_back; j < it; ++j)
+                    if (!mbar_wait(smem_u32(&ctrl->scale_full[j % G_SCALE_RING]), (j / G_SCALE_RING) & 1, &zero, limit))
                         atomicCAS(g.status, DEV_OK, DEV_TIMEOUT_DRAIN);
             }
         } else if ((warp == 1 || warp == 2) && lane == 0) {
@@ -206,12 +228,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint64_t a_desc = umma_desc_sw128(a_addr);
                     const uint64_t b_desc = umma_desc_sw128(a_addr + G_A_BYTES);
                     const uint32_t d_tmem = tmem_base + b * G_TILE_N;
-                    if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag)) {
+                    if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, limit)) {
                         raise(ctrl, g.status, DEV_TIMEOUT_MMA_SMEM);
                         ok = false;
                         break;
                     }
-                    if (!mbar_wait(smem_u32(&ctrl->tmem_empty[b]), bph ^ 1, abort_flag)) {
+                    if (!mbar_wait(smem_u32(&ctrl->tmem_empty[b]), bph ^ 1, abort_flag, limit)) {
                         raise(ctrl, g.status, DEV_TIMEOUT_MMA_TMEM);
                         ok = false;
                         break;
@@ -226,7 +248,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (!ok || *abort_flag) {  // let issued MMAs retire before TMEM is released
                 umma_commit(smem_u32(&ctrl->drain_bar[mine]));
                 int zero = 0;
-                mbar_wait(smem_u32(&ctrl->drain_bar[mine]), 0, &zero);
+                mbar_wait(smem_u32(&ctrl->drain_bar[mine]), 0, &zero, limit);
             }
         }
     } else {
@@ -244,8 +266,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tile_iter) {
             const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
-            const int e = __ldg(g.tile_expert + m_tile);
-            const int rows_valid = __ldg(g.tile_rows + m_tile);
+            const int e = __ldcg(g.tile_expert + m_tile);
+            const int rows_valid = __ldcg(g.tile_rows + m_tile);
             const size_t row = static_cast<size_t>(m_tile) * TILE_M + r_in_tile;
             const int sblocks = g.w_rows_per_expert / 128;
             // weight-scale rows of this thread's first / second 64 columns
@@ -270,17 +292,24 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     s1 = __ldg(ws1 + kb + 1);
                 }
                 const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1, buf = it & 1;
-                if (!mbar_wait(smem_u32(&ctrl->done[s]), ph, abort_flag)) {
-                    raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                // The activation scale of this K-block comes first: its copy landed with (or before) the
+                // operand tiles, i.e. long before the MMAs on them end, so this wait and the load are off the
+                // accumulator hand-over.  (The ring's own barriers are needed for that: on full[s] this warp
+                // can be lapped by a whole phase, which a parity wait cannot tell apart.)
+                const uint32_t sl = it % G_SCALE_RING;
+                if (!mbar_wait_warp(smem_u32(&ctrl->scale_full[sl]), (it / G_SCALE_RING) & 1, abort_flag, lane, limit)) {
+                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                    ok = false;
+                    break;
+                }
+                const float sa = ld_shared_f32(scale_ring + sl * TILE_M + r_in_tile);
+                const float f0 = sa * w0, f1 = sa * w1;
+                if (!mbar_wait_warp(smem_u32(&ctrl->done[s]), ph, abort_flag, lane, limit)) {
+                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                // The MMA of this K-block has finished, hence its stage -- A, B and the scales -- had landed.
-                // (Waiting on full[s] here instead, to fetch the scale earlier, would be wrong: this warp may
-                // be lapped by a whole phase of that barrier, and a parity wait cannot tell the difference.)
-                const float sa = ld_shared_f32(scale_ring + (it % G_SCALE_RING) * TILE_M + r_in_tile);
-                const float f0 = sa * w0, f1 = sa * w1;
                 // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
                 const uint32_t col = t_lane + buf * G_TILE_N;
                 float v[64];
@@ -318,8 +347,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 amax_x[(par * 2 + half) * TILE_M + r_in_tile] = amax;
                 const uint32_t xbar = smem_u32(&ctrl->amax_bar[par]);
                 mbar_arrive(xbar);
-                if (!mbar_wait(xbar, (tile_iter >> 1) & 1, abort_flag)) {
-                    raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                if (!mbar_wait_warp(xbar, (tile_iter >> 1) & 1, abort_flag, lane, limit)) {
+                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
                     break;
                 }
                 amax = fmaxf(amax,

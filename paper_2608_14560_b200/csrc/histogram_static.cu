@@ -20,6 +20,7 @@ constexpr int STATIC_MAX_BLOCKS =
 // loads the library until the process exits.  In host code this name is only a handle for
 // cudaGetSymbolAddress; the device address is looked up once per device below.
 static __device__ __align__(256) int g_block_hist[STATIC_MAX_BLOCKS * P_MAX_LOCAL];
+static_assert(STATIC_MAX_BLOCKS * P_MAX_LOCAL * sizeof(int) == 65536, "the documented size of the fixed scratch");
 
 constexpr int MAX_DEVICES = 64;
 int* g_block_hist_addr[MAX_DEVICES] = {};

@@ -92,6 +92,8 @@ struct moe_fp8_handle_s {
     const void* w2_cached;
     bool stage_timing;
     bool stage_times_valid;
+    int fault_skip_it;         // test hook, see moe_fp8_debug_set_fault
+    long long fault_wait_limit;
     cudaEvent_t ev[9];
 };
 
@@ -160,6 +162,11 @@ const char* const STAGE_NAMES[NUM_STAGES] = {"route_topk", "count", "scan", "pla
                                              "gemm1_swiglu_quant", "gemm2", "combine"};
 
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+// Test hook: the routing stage's sigmoid on arbitrary inputs.
+__global__ void sigmoid_export_kernel(int n, const float* __restrict__ x, float* __restrict__ y) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) y[i] = sigmoid_fixed(x[i]);
+}
 
 // Debug: canonical row r -> padded row, then copy that row's intermediate results.
 __global__ void export_rows_kernel(int E_loc, int I, int H, int row_cap, const int* __restrict__ expert_offset,
@@ -240,6 +247,8 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     h->cfg = *cfg;
     h->L = make_layout(*cfg);
     h->sm_count = sms;
+    h->fault_skip_it = -1;
+    h->fault_wait_limit = WAIT_LIMIT_CLOCKS;
     h->encode = reinterpret_cast<EncodeTiledFn>(fn);
     *out = h;
     return MOE_FP8_OK;
@@ -257,8 +266,11 @@ size_t moe_fp8_workspace_bytes(moe_fp8_handle_t h) { return h ? h->L.total : 0; 
 int moe_fp8_set_workspace(moe_fp8_handle_t h, void* ws, size_t bytes) {
     if (!h || !ws || (reinterpret_cast<uintptr_t>(ws) % WS_ALIGN) != 0) return MOE_FP8_ERR_BAD_ARG;
     if (bytes < h->L.total) return MOE_FP8_ERR_NO_WORKSPACE;
-    // the device status word and the ticket counter of route_permute_kernel start at zero
+    // The device status word and the ticket counter of route_permute_kernel start at zero.  A memset of device
+    // memory is asynchronous to the host and a forward may follow on a non-blocking stream, which does not
+    // order itself behind the default stream: wait for it here.
     cudaError_t e = cudaMemset(static_cast<uint8_t*>(ws) + h->L.status, 0, 2 * sizeof(int));
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->ws = static_cast<uint8_t*>(ws);
     h->ws_bytes = bytes;
@@ -331,15 +343,22 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     auto mark = [&]() {
         if (h->stage_timing) cudaEventRecord(h->ev[ev_i++], stream);
     };
+    // The first launch that fails ends the call: nothing further is enqueued behind it.
+    cudaError_t lerr = cudaSuccess;
+#define MOE_LAUNCH(...)                                   \
+    do {                                                  \
+        lerr = launch(__VA_ARGS__);                       \
+        if (lerr != cudaSuccess) return cuda_fail(h, lerr); \
+        ++launches;                                       \
+    } while (0)
     h->stage_times_valid = false;
     mark();
 
     if (T <= P_TAIL_MAX_TOKENS) {  // routing in parallel blocks, the last one to finish does stage 2
         const int grid = min((T + 7) / 8, h->sm_count * 8);
-        launch(route_permute_kernel, grid, P_TAIL_THREADS, route_permute_smem_bytes(T, EL), stream, false, T, EL,
-               local_expert_offset, row_cap, router_logits, static_cast<const __nv_bfloat16*>(routing_bias),
-               scaling_factor, topk_idx, topk_w, m, status + 1, status);
-        ++launches;
+        MOE_LAUNCH(route_permute_kernel, grid, P_TAIL_THREADS, route_permute_smem_bytes(T, EL), stream, false, T, EL,
+                   local_expert_offset, row_cap, router_logits, static_cast<const __nv_bfloat16*>(routing_bias),
+                   scaling_factor, topk_idx, topk_w, m, status + 1, status);
         mark();
         mark();
         mark();
@@ -347,28 +366,25 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     } else {
         {  // stage 1: routing
             const int grid = min((T + 7) / 8, h->sm_count * 8);
-            launch(route_topk_kernel, grid, 256, 0, stream, false, T, router_logits,
-                   static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w, status);
-            ++launches;
+            MOE_LAUNCH(route_topk_kernel, grid, 256, 0, stream, false, T, router_logits,
+                       static_cast<const __nv_bfloat16*>(routing_bias), scaling_factor, topk_idx, topk_w, status);
             mark();
         }
         // stage 2: histogram, scan, placement
-        launch(count_kernel, nblk, P_TOKENS_PER_BLOCK, 0, stream, pdl, T, EL, local_expert_offset,
-               static_cast<const int*>(topk_idx), m.block_hist);
+        MOE_LAUNCH(count_kernel, nblk, P_TOKENS_PER_BLOCK, 0, stream, pdl, T, EL, local_expert_offset,
+                   static_cast<const int*>(topk_idx), m.block_hist);
         mark();
-        launch(scan_kernel, 1, P_MAX_LOCAL, 0, stream, pdl, nblk, EL, m);
+        MOE_LAUNCH(scan_kernel, 1, P_MAX_LOCAL, 0, stream, pdl, nblk, EL, m);
         mark();
-        launch(place_kernel, nblk, P_TOKENS_PER_BLOCK, 0, stream, pdl, T, EL, local_expert_offset, row_cap,
-               static_cast<const int*>(topk_idx), m, status);
+        MOE_LAUNCH(place_kernel, nblk, P_TOKENS_PER_BLOCK, 0, stream, pdl, T, EL, local_expert_offset, row_cap,
+                   static_cast<const int*>(topk_idx), m, status);
         mark();
-        launches += 3;
     }
     {  // stage 2, continued: gather
         const long long row_bound = static_cast<long long>(T) * 8 + static_cast<long long>(EL) * (TILE_M - 1);
         const int grid = static_cast<int>(std::min<long long>((row_bound + 7) / 8, h->sm_count * 8LL));
-        launch(gather_rows_kernel, grid, 256, 0, stream, pdl, H, row_cap, c.hidden_scale_layout, T,
-               static_cast<const uint8_t*>(hidden_fp8), hidden_scale, m, a1, a1_scale_t);
-        ++launches;
+        MOE_LAUNCH(gather_rows_kernel, grid, 256, 0, stream, pdl, H, row_cap, c.hidden_scale_layout, T,
+                   static_cast<const uint8_t*>(hidden_fp8), hidden_scale, m, a1, a1_scale_t);
         mark();
     }
     {  // stage 3a: GEMM1 + SwiGLU + re-quantisation
@@ -389,9 +405,10 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         g.out_fp8 = a2;
         g.out_scale_t = a2_scale_t;
         g.status = status;
-        launch(grouped_gemm_kernel<1>, h->sm_count, G_THREADS, G_SMEM_BYTES, stream, pdl, h->tm_a1, h->tm_w13,
-               h->tm_a2_store, g);
-        ++launches;
+        g.wait_limit = h->fault_wait_limit;
+        g.fault_skip_it = h->fault_skip_it;
+        MOE_LAUNCH(grouped_gemm_kernel<1>, h->sm_count, G_THREADS, G_SMEM_BYTES, stream, pdl, h->tm_a1, h->tm_w13,
+                   h->tm_a2_store, g);
         mark();
     }
     {  // stage 3b: GEMM2
@@ -409,24 +426,40 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         g.w_scale = w2_scale;
         g.out_bf16 = y;
         g.status = status;
-        launch(grouped_gemm_kernel<2>, h->sm_count, G_THREADS, G_SMEM_BYTES, stream, pdl, h->tm_a2, h->tm_w2,
-               h->tm_a2_store, g);
-        ++launches;
+        g.wait_limit = h->fault_wait_limit;
+        g.fault_skip_it = -1;
+        MOE_LAUNCH(grouped_gemm_kernel<2>, h->sm_count, G_THREADS, G_SMEM_BYTES, stream, pdl, h->tm_a2, h->tm_w2,
+                   h->tm_a2_store, g);
         mark();
     }
     {  // stage 4: weighted combine back to token order
         const int grid = min(T, h->sm_count * 16);
-        launch(combine_kernel, grid, 256, 0, stream, pdl, T, H, static_cast<const int*>(m.slot_to_row),
-               static_cast<const float*>(topk_w), reinterpret_cast<const uint8_t*>(y),
-               static_cast<__nv_bfloat16*>(out));
-        ++launches;
+        MOE_LAUNCH(combine_kernel, grid, 256, 0, stream, pdl, T, H, static_cast<const int*>(m.slot_to_row),
+                   static_cast<const float*>(topk_w), reinterpret_cast<const uint8_t*>(y),
+                   static_cast<__nv_bfloat16*>(out));
         mark();
     }
+#undef MOE_LAUNCH
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_launches = launches;
     h->stage_times_valid = h->stage_timing;
     return MOE_FP8_OK;
+}
+
+int moe_fp8_debug_set_fault(moe_fp8_handle_t h, int skip_iteration, long long wait_clocks) {
+    if (!h || wait_clocks < 0) return MOE_FP8_ERR_BAD_ARG;
+    h->fault_skip_it = skip_iteration < 0 ? -1 : skip_iteration;
+    h->fault_wait_limit = wait_clocks == 0 ? WAIT_LIMIT_CLOCKS : wait_clocks;
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_debug_sigmoid(int n, const float* x, float* y, void* stream_v) {
+    if (n < 0 || (n > 0 && (!x || !y))) return MOE_FP8_ERR_BAD_ARG;
+    if (n == 0) return MOE_FP8_OK;
+    sigmoid_export_kernel<<<(n + 255) / 256 > 1184 ? 1184 : (n + 255) / 256, 256, 0,
+                            static_cast<cudaStream_t>(stream_v)>>>(n, x, y);
+    return cudaGetLastError() == cudaSuccess ? MOE_FP8_OK : MOE_FP8_ERR_CUDA;
 }
 
 int moe_fp8_set_stage_timing(moe_fp8_handle_t h, int enable) {

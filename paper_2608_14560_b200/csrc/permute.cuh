@@ -34,15 +34,17 @@ struct PermuteMeta {
 
 // Bit t of mask[e] says: token t of this block routes to local expert e.  The
 // popcount below a token's bit is its stable rank inside the block.
+// topk_idx was written by the kernel before this one, which may still be resident (programmatic dependent
+// launch): it is read with coherent (.cg) loads, never through the read-only path.
 __device__ __forceinline__ void build_block_masks(uint32_t (*mask)[P_TOKENS_PER_BLOCK / 32], int T, int E_loc,
-                                                  int off, const int* __restrict__ topk_idx) {
+                                                  int off, const int* topk_idx) {
     for (int i = threadIdx.x; i < E_loc * (P_TOKENS_PER_BLOCK / 32); i += blockDim.x)
         (&mask[0][0])[i] = 0u;
     __syncthreads();
     const int t = blockIdx.x * P_TOKENS_PER_BLOCK + threadIdx.x;
     if (t < T) {
-        const int4 a = reinterpret_cast<const int4*>(topk_idx)[2 * t];
-        const int4 b = reinterpret_cast<const int4*>(topk_idx)[2 * t + 1];
+        const int4 a = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t);
+        const int4 b = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t + 1);
         const int ids[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -54,7 +56,7 @@ __device__ __forceinline__ void build_block_masks(uint32_t (*mask)[P_TOKENS_PER_
 }
 
 __global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) count_kernel(int T, int E_loc, int off,
-                                                                   const int* __restrict__ topk_idx,
+                                                                   const int* topk_idx,
                                                                    int* __restrict__ block_hist) {
     pdl_launch_dependents();
     pdl_wait();
@@ -117,7 +119,7 @@ __global__ void __launch_bounds__(P_MAX_LOCAL) scan_kernel(int nblk, int E_loc, 
 }
 
 __global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) place_kernel(int T, int E_loc, int off, int row_cap,
-                                                                   const int* __restrict__ topk_idx, PermuteMeta m,
+                                                                   const int* topk_idx, PermuteMeta m,
                                                                    int* __restrict__ status) {
     pdl_launch_dependents();
     pdl_wait();
@@ -128,7 +130,7 @@ __global__ void __launch_bounds__(P_TOKENS_PER_BLOCK) place_kernel(int T, int E_
     const int word = threadIdx.x >> 5, bit = threadIdx.x & 31;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const int e = topk_idx[t * 8 + j] - off;
+        const int e = __ldcg(topk_idx + t * 8 + j) - off;
         int prow = -1;
         if (e >= 0 && e < E_loc) {
             int rank = __popc(mask[e][word] & ((1u << bit) - 1u));
@@ -191,6 +193,12 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
         const int n = atomicAdd(ticket, 1);
         s_last = (n == static_cast<int>(gridDim.x) - 1);
         if (s_last) *ticket = 0;
+        // A counter that did not start at zero (somebody wrote into the workspace) would leave this forward
+        // without a last block and with stale tables: say so instead of returning them silently.
+        if (n < 0 || n >= static_cast<int>(gridDim.x)) {
+            atomicExch(status, DEV_BAD_TICKET);
+            *ticket = 0;
+        }
     }
     __syncthreads();
     if (!s_last) return;

@@ -16,7 +16,11 @@ enum : int {
     DEV_TIMEOUT_EPILOGUE = 4,  // epilogue never saw a finished accumulator buffer
     DEV_TIMEOUT_DRAIN = 5,     // in-flight copies did not land during abort
     DEV_BAD_ROW = 6,           // a computed row index fell outside its buffer
+    DEV_BAD_TICKET = 7,        // the last-block ticket counter in the workspace was not zero at launch
 };
+
+// Clocks a bounded wait spins before it gives up (about a second at 2 GHz).
+constexpr long long WAIT_LIMIT_CLOCKS = 1ll << 31;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -55,9 +59,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
-// Bounded wait: gives up after ~2^31 clocks (about a second) or as soon as another
-// role of the CTA raised `*abort_flag`.  Returns false when it gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait: gives up after `limit` clocks or as soon as another role of the CTA
+// raised `*abort_flag`.  Returns false when it gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit = WAIT_LIMIT_CLOCKS) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
@@ -65,8 +70,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > (1ll << 31)) return false;
+        if (clock64() - t0 > limit) return false;
     }
+}
+// The same wait for a whole (converged) warp: lane 0 polls and decides, every lane gets its verdict, so the
+// warp stays converged whether the wait succeeded or gave up.  The __syncwarp orders lane 0's acquire of the
+// barrier phase before the other lanes' later accesses.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int lane,
+                                               long long limit = WAIT_LIMIT_CLOCKS) {
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, limit) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();
+    return ok != 0;
 }
 
 // Plain (weak) 32-bit shared-memory load that the compiler may neither cache nor move: a C++ volatile
@@ -190,11 +206,13 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&w)[8]) {
                  ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                  : "memory");
 }
-// 32-byte global load through the read-only path.
-__device__ __forceinline__ void ld_global_nc_v8(const void* p, uint32_t (&w)[8]) {
-    asm volatile("ld.global.nc.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+// 32-byte global load, not kept in L1.  A coherent load, not the read-only (.nc) path: the data may have been
+// written by the kernel before this one while this kernel was already resident (programmatic dependent launch).
+__device__ __forceinline__ void ld_global_v8(const void* p, uint32_t (&w)[8]) {
+    asm volatile("ld.global.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                  : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
-                 : "l"(p));
+                 : "l"(p)
+                 : "memory");
 }
 
 // ---- registers --------------------------------------------------------------

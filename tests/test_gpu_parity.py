@@ -178,26 +178,96 @@ def _sample(T, n, seed):
     return np.sort(np.random.default_rng(seed).choice(T, n, replace=False)).astype(np.int32)
 
 
-@pytest.mark.parametrize("cfg,n_sample", [(0, 8), (1, 64), (2, 256), (3, 40)])
-def test_benchmark_workloads_32_local_experts(cuda_device, cfg, n_sample):
+# Output: every token up to T = 1024, else 256 random tokens.  Per-slot rows (re-quantised intermediate and
+# down-projection row): on the large workloads every row of the first and the last row tile of the largest
+# expert segment, of the smallest non-empty segment and of the first tile of a median one -- whole tiles at the
+# full K depth, on CTAs that have walked many tiles before them.
+@pytest.mark.parametrize("cfg,n_sample,rows", [(0, 8, True), (1, 64, True), (2, 1024, "tiles"), (3, 256, "tiles")])
+def test_benchmark_workloads_32_local_experts(cuda_device, cfg, n_sample, rows):
     wl = syn.CONFIGS[cfg]
-    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(wl.tokens, n_sample, cfg))
+    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(wl.tokens, n_sample, cfg), check_rows=rows)
     print(wl.name, st)
 
 
-@pytest.mark.parametrize("tokens,n_sample", [(7, 7), (54, 54), (14107, 32)])
-def test_token_counts_quoted_in_the_paper(cuda_device, tokens, n_sample):
+@pytest.mark.parametrize("tokens,n_sample,rows", [(7, 7, True), (54, 54, True), (14107, 256, "tiles")])
+def test_token_counts_quoted_in_the_paper(cuda_device, tokens, n_sample, rows):
     # the paper's table of workload regimes (short / median / long) quotes one latency each for T = 7, 54 and
     # 14107 tokens with 32 local experts
     base = syn.CONFIGS[1]
     wl = syn.Workload(f"dsv3_T{tokens}_E32", tokens, base.dims, base.seed, base.local_expert_offset,
                       base.scaling_factor, base.skew)
-    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(tokens, n_sample, tokens))
+    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(tokens, n_sample, tokens), check_rows=rows)
     print(wl.name, st)
 
 
 def test_benchmark_workload_all_256_experts_local(cuda_device):
     wl = syn.CONFIGS[4]
-    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(wl.tokens, 24, 4))
+    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(wl.tokens, 256, 4), check_rows="tiles")
     assert st["S"] == wl.tokens * 8
     print(wl.name, st)
+
+
+def test_routing_on_logits_far_outside_the_unit_range(cuda_device):
+    # the fixed-operation sigmoid on its clamped tails and at large |logit|: indices and weights of the
+    # kernel must equal the oracle's bit for bit there too, not only on N(0,1) logits
+    wl = _wl(256, seed=31)
+    inp = syn.make_inputs(wl, cuda_device)
+    g = torch.Generator(device=cuda_device)
+    g.manual_seed(77)
+    mags = torch.tensor([8.0, 20.0, 87.0, 88.0, 100.0, 1e4, 0.015625, 3.0], device=cuda_device)
+    pick = torch.randint(0, len(mags), inp["router_logits"].shape, generator=g, device=cuda_device)
+    sign = torch.randint(0, 2, inp["router_logits"].shape, generator=g, device=cuda_device) * 2.0 - 1.0
+    inp["router_logits"] = (mags[pick] * sign).contiguous()
+    run_and_compare(wl, cuda_device, inp=inp)
+    # a dense sweep of the benchmark's 1/64 grid over [-32, 32] and of large magnitudes, one value per expert column
+    T = 4096 // 256 * 2
+    grid = (torch.arange(-2048, 2048, device=cuda_device, dtype=torch.float32) / 64.0).view(-1, 256)
+    big = (torch.arange(-2048, 2048, device=cuda_device, dtype=torch.float32) / 16.0).view(-1, 256)
+    wl2 = _wl(T, seed=32)
+    inp2 = syn.make_inputs(wl2, cuda_device)
+    inp2["router_logits"] = torch.cat([grid, big]).contiguous()
+    run_and_compare(wl2, cuda_device, inp=inp2)
+
+
+def test_device_sigmoid_bits_equal_the_oracle(cuda_device):
+    # every point of the benchmark's logit grid (k/64, |k| <= 2048), the clamp boundaries and 2^20 random
+    # floats over the whole finite range: the kernel's sigmoid and the oracle's agree in every bit
+    from paper_2608_14560_b200 import binding
+    rng = np.random.default_rng(11)
+    grid = (np.arange(-2048, 2049) / 64.0).astype(np.float32)
+    edge = np.float32([0.0, -0.0, 87.0, -87.0, 88.0, -88.0, 88.5, -88.5, 100.0, -100.0, 1e4, -1e4, 3e38, -3e38,
+                       1e-30, -1e-30, 1e-45, 0.34657359, -0.34657359])
+    rnd_bits = rng.integers(0, 1 << 32, 1 << 20, dtype=np.uint64).astype(np.uint32)
+    rnd = rnd_bits.view(np.float32)
+    rnd = rnd[np.isfinite(rnd)]
+    mid = (rng.standard_normal(1 << 18) * 6.0).astype(np.float32)
+    x = np.concatenate([grid, edge, rnd, mid]).astype(np.float32)
+    got = binding.debug_sigmoid(torch.from_numpy(x).to(cuda_device)).cpu().numpy()
+    want = oracle.sigmoid(x)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), \
+        f"{(got.view(np.uint32) != want.view(np.uint32)).sum()} of {x.size} sigmoid values differ"
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable(cuda_device):
+    # The copy producer of GEMM1 is told to stop before its third pipeline stage and every wait limit is
+    # shortened to 2^20 clocks: the consumers' waits give up, the kernel returns with a time-out code in the
+    # status word (nothing traps, nothing spins without a bound), and the next forward on the same handle,
+    # with the hook off again, is bit-identical to a forward on a fresh handle.
+    wl = _wl(300, seed=41)
+    inp = syn.make_inputs(wl, cuda_device)
+    fresh = make_engine(wl, cuda_device)
+    want = fresh.forward(inp).clone()
+    torch.cuda.synchronize()
+    fresh.close()
+    eng = make_engine(wl, cuda_device)
+    eng.debug_set_fault(skip_iteration=2, wait_clocks=1 << 20)
+    eng.forward(inp)
+    torch.cuda.synchronize()
+    assert 1 <= eng.status() <= 5, f"expected a time-out code, got {eng.status()}"
+    eng.debug_set_fault(-1, 0)
+    got = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert eng.status() == 0
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    run_and_compare(wl, cuda_device, inp=inp, eng=eng)
+    eng.close()

@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2608_14560_b200 import binding
 from paper_2608_14560_b200 import synthetic as syn
 
@@ -46,6 +47,29 @@ def test_static_histogram_matches_workspace_path_on_two_calls_in_a_row(cuda_devi
         assert torch.equal(count, want_count)
         assert torch.equal(offset, want_offset)
         assert int(offset[-1]) == int(want_count.sum())
+        # and against the CPU oracle's permutation of the same routing indices
+        perm = oracle.permute(idx.cpu().numpy(), wl.local_expert_offset, el)
+        assert np.array_equal(count.cpu().numpy(), perm["count"])
+        assert np.array_equal(offset.cpu().numpy(), perm["offset"])
+
+
+def test_static_histogram_at_its_capacity_then_a_small_call(cuda_device):
+    # the largest call the fixed array admits (every one of its 64 x 256 entries is used), checked against a
+    # library histogram; the small call after it must not see anything the large one left behind
+    g = torch.Generator(device=cuda_device)
+    g.manual_seed(9)
+    for T, el, off in [(binding.STATIC_HISTOGRAM_MAX_TOKENS, 256, 0), (5, 7, 100)]:
+        # 8 distinct experts per token, as routing produces them
+        idx = torch.rand(T, 256, generator=g, device=cuda_device).argsort(dim=1)[:, :8].to(torch.int32).contiguous()
+        count = torch.full((el,), -7, dtype=torch.int32, device=cuda_device)
+        offset = torch.full((el + 1,), -7, dtype=torch.int32, device=cuda_device)
+        assert binding.expert_histogram_static(idx, off, el, count, offset) == binding.OK
+        torch.cuda.synchronize()
+        local = idx.long().flatten() - off
+        local = local[(local >= 0) & (local < el)]
+        want = torch.bincount(local, minlength=el).to(torch.int32)
+        assert torch.equal(count, want)
+        assert torch.equal(offset[1:], torch.cumsum(want, 0).to(torch.int32)) and int(offset[0]) == 0
 
 
 def test_static_histogram_rejects_sizes_beyond_its_capacity(cuda_device):
