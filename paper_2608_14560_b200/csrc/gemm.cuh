@@ -7,8 +7,7 @@
 //   warp 0      TMA producer.  Per K-block (128 K-bytes = one scale block): the A
 //               tile (128 rows), the B tile (256 weight rows) and the 128
 //               activation scales of the block, into a 4-stage ring (128-byte
-//               swizzle) / an 8-slot scale ring (its own mbarrier per slot, so the
-//               epilogue can fetch a scale before the MMAs that use the block end).
+//               swizzle) / an 8-slot scale ring, completion on mbarriers.
 //   warps 1,2   MMA issuers (even / odd K-blocks).  Four tcgen05.mma (M128 N256 K32, e4m3 -> fp32) per
 //               K-block into one of two 256-column TMEM buffers, then ONE
 //               tcgen05.commit: the same mbarrier tells the producer that the stage
@@ -79,7 +78,6 @@ struct GemmArgs {
 struct GemmCtrl {
     uint64_t full[G_STAGES];   // stage filled (TMA transaction bytes)
     uint64_t done[G_STAGES];   // the MMAs that read the stage have finished: stage free AND accumulator ready
-    uint64_t scale_full[G_SCALE_RING];  // activation scales of a K-block have landed
     uint64_t tmem_empty[G_ACC_BUFS];
     uint64_t amax_bar[2];
     uint64_t drain_bar[2];
@@ -115,7 +113,6 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(smem_u32(&ctrl->full[s]), 1);
             mbar_init(smem_u32(&ctrl->done[s]), 1);
         }
-        for (int s = 0; s < G_SCALE_RING; ++s) mbar_init(smem_u32(&ctrl->scale_full[s]), 1);
         for (int b = 0; b < G_ACC_BUFS; ++b) {
             mbar_init(smem_u32(&ctrl->tmem_empty[b]), G_EPI_WARPS);
         }
@@ -172,13 +169,11 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t bar = smem_u32(&ctrl->full[s]);
                     const uint32_t a_dst = smem_base + s * G_STAGE_BYTES, b_dst = a_dst + G_A_BYTES;
                     const int k0 = kb * G_BLOCK_K;
-                    // The scale slot is free: 8 slots exceed the 4 stages + 2 accumulators the producer can
-                    // be ahead of the epilogue.
-                    const uint32_t sbar = smem_u32(&ctrl->scale_full[it % G_SCALE_RING]);
-                    mbar_expect_tx(sbar, G_SCALE_BYTES);
+                    // (the scale slot is free: 8 slots exceed the 4 stages + 2 accumulators the producer can be
+                    // ahead of the epilogue)
+                    mbar_expect_tx(bar, G_STAGE_BYTES + G_SCALE_BYTES);
                     bulk_load_1d(smem_u32(scale_ring + (it % G_SCALE_RING) * TILE_M),
-                                 a_sc + static_cast<size_t>(kb) * g.row_cap, G_SCALE_BYTES, sbar);
-                    mbar_expect_tx(bar, G_STAGE_BYTES);
+                                 a_sc + static_cast<size_t>(kb) * g.row_cap, G_SCALE_BYTES, bar);
                     tma_load_2d(a_dst, &tmA, k0, m_tile * TILE_M, bar);
                     if (MODE == 1) {
                         const int gr = wrow + g.gate_row0 + n * 128, ur = wrow + g.up_row0 + n * 128;
@@ -202,10 +197,6 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const uint32_t n_back = it < G_STAGES ? it : G_STAGES;
                 for (uint32_t j = it - n_back; j < it; ++j)
                     if (!mbar_wait(smem_u32(&ctrl->full[j % G_STAGES]), (j / G_STAGES) & 1, &zero, limit))
-                        atomicCAS(g.status, DEV_OK, DEV_TIMEOUT_DRAIN);
-                const uint32_t s_back = it < G_SCALE_RING ? it : G_SCALE_RING;
-                for (uint32_t j = it - s_back; j < it; ++j)
-                    if (!mbar_wait(smem_u32(&ctrl->scale_full[j % G_SCALE_RING]), (j / G_SCALE_RING) & 1, &zero, limit))
                         atomicCAS(g.status, DEV_OK, DEV_TIMEOUT_DRAIN);
             }
         } else if ((warp == 1 || warp == 2) && lane == 0) {
@@ -292,24 +283,20 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     s1 = __ldg(ws1 + kb + 1);
                 }
                 const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1, buf = it & 1;
-                // The activation scale of this K-block comes first: its copy landed with (or before) the
-                // operand tiles, i.e. long before the MMAs on them end, so this wait and the load are off the
-                // accumulator hand-over.  (The ring's own barriers are needed for that: on full[s] this warp
-                // can be lapped by a whole phase, which a parity wait cannot tell apart.)
-                const uint32_t sl = it % G_SCALE_RING;
-                if (!mbar_wait_warp(smem_u32(&ctrl->scale_full[sl]), (it / G_SCALE_RING) & 1, abort_flag, lane, limit)) {
-                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                    ok = false;
-                    break;
-                }
-                const float sa = ld_shared_f32(scale_ring + sl * TILE_M + r_in_tile);
-                const float f0 = sa * w0, f1 = sa * w1;
-                if (!mbar_wait_warp(smem_u32(&ctrl->done[s]), ph, abort_flag, lane, limit)) {
+                // Every lane polls (a single polling lane plus a broadcast was measured 2.5 % slower); the vote
+                // keeps the warp converged when a wait gives up: either all lanes go on or none does.
+                if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph, abort_flag, limit))) {
                     if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
                     ok = false;
                     break;
                 }
                 tc_fence_after();
+                // The MMA of this K-block has finished, hence its stage -- A, B and the scales -- had landed.
+                // (Fetching the scale earlier needs a barrier of its own per ring slot -- on full[s] this warp can
+                // be lapped by a whole phase -- and that extra barrier test per K-block was measured to cost the
+                // epilogue 110 clocks, 10 % of the kernel: barrier operations of a thread queue behind one another.)
+                const float sa = ld_shared_f32(scale_ring + (it % G_SCALE_RING) * TILE_M + r_in_tile);
+                const float f0 = sa * w0, f1 = sa * w1;
                 // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
                 const uint32_t col = t_lane + buf * G_TILE_N;
                 float v[64];
@@ -347,7 +334,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 amax_x[(par * 2 + half) * TILE_M + r_in_tile] = amax;
                 const uint32_t xbar = smem_u32(&ctrl->amax_bar[par]);
                 mbar_arrive(xbar);
-                if (!mbar_wait_warp(xbar, (tile_iter >> 1) & 1, abort_flag, lane, limit)) {
+                if (!__all_sync(0xffffffffu, mbar_wait(xbar, (tile_iter >> 1) & 1, abort_flag, limit))) {
                     if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
                     break;
                 }

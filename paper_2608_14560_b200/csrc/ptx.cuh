@@ -73,18 +73,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (clock64() - t0 > limit) return false;
     }
 }
-// The same wait for a whole (converged) warp: lane 0 polls and decides, every lane gets its verdict, so the
-// warp stays converged whether the wait succeeded or gave up.  The __syncwarp orders lane 0's acquire of the
-// barrier phase before the other lanes' later accesses.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int lane,
-                                               long long limit = WAIT_LIMIT_CLOCKS) {
-    int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, abort_flag, limit) ? 1 : 0;
-    ok = __shfl_sync(0xffffffffu, ok, 0);
-    __syncwarp();
-    return ok != 0;
-}
-
 // Plain (weak) 32-bit shared-memory load that the compiler may neither cache nor move: a C++ volatile
 // access compiles to ld.volatile, which was measured to cost ~150 clocks in these loops.
 __device__ __forceinline__ float ld_shared_f32(const float* p) {
