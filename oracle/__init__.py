@@ -99,6 +99,42 @@ def sigmoid(x) -> np.ndarray:
     return np.array([f(float(v)) for v in x.ravel()], dtype=np.float32).reshape(x.shape)
 
 
+def router_logits(x_bf16, w_bf16) -> np.ndarray:
+    """Router projection in the fixed fp32 summation order: x [T,H], w [E,H] bf16 bits -> logits [T,E] fp32."""
+    x = _c(x_bf16, np.uint16)
+    w = _c(w_bf16, np.uint16)
+    T, H = x.shape
+    E = w.shape[0]
+    assert w.shape[1] == H
+    out = np.empty((T, E), np.float32)
+    _check(lib().moe_ref_router_logits(C.c_int(T), C.c_int(H), C.c_int(E), _p(x, C.c_uint16), _p(w, C.c_uint16),
+                                       _p(out, C.c_float)), "router_logits")
+    return out
+
+
+def quantize_rows(x_bf16):
+    """Input-side activation quantisation: x [T,H] bf16 bits -> (codes uint8 [T,H], scale fp32 [T,H/128])."""
+    x = _c(x_bf16, np.uint16)
+    T, H = x.shape
+    q = np.empty((T, H), np.uint8)
+    s = np.empty((T, H // 128), np.float32)
+    _check(lib().moe_ref_quantize_rows(C.c_int(T), C.c_int(H), _p(x, C.c_uint16), _p(q, C.c_uint8), _p(s, C.c_float)),
+           "quantize_rows")
+    return q, s
+
+
+def forward_from_hidden(inp: dict, n_group: int, topk_group: int, top_k: int, tokens=None, **kw):
+    """The layer starting from bf16 hidden states: router projection, input quantisation, then forward().
+    inp carries hidden_bf16 [T,H] and router_weight [E,H] (bf16 bits) instead of hidden_fp8 / hidden_scale /
+    router_logits.  -> forward()'s dict plus the logits, codes and scales it was given."""
+    logits = router_logits(inp["hidden_bf16"], inp["router_weight"])
+    q, s = quantize_rows(inp["hidden_bf16"])
+    full = dict(inp, hidden_fp8=q, hidden_scale=s, router_logits=logits)
+    res = forward(full, n_group, topk_group, top_k, tokens=tokens, **kw)
+    res.update(router_logits=logits, hidden_fp8=q, hidden_scale=s)
+    return res
+
+
 def route(logits, bias_bf16, n_group, topk_group, top_k, scaling, want_sig=False):
     """-> (topk_idx [T,K] int32, topk_w [T,K] fp32[, sig [T,E]])."""
     logits = _c(logits, np.float32)

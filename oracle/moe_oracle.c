@@ -18,6 +18,10 @@
  * Pins (tests that do not pass through this file's own formulas):
  *   - FP8/bf16 codecs: every code against the library conversion of PyTorch.
  *   - expdet/sigmoid: within 2 ulp of the fp64 library exp.
+ *   - router projection: fp64 library matmul within the fp32 error bound, a
+ *     hand-worked case with exact integer sums, and a hand-worked case whose
+ *     value depends on the summation order; input quantisation: the library
+ *     cast of PyTorch, bit for bit.
  *   - routing: closed forms (uniform logits; planted winners), a hand-worked
  *     miniature, a brute-force full sort, the weight-sum invariant.
  *   - permutation: bijection + a library stable sort.
@@ -142,6 +146,77 @@ float moe_ref_expdet(float x)
 float moe_ref_sigmoid(float x)
 {
     return 1.0f / (1.0f + moe_ref_expdet(-x));
+}
+
+/* Router projection: the "lightweight linear projection" that produces the
+ * routing scores in stage 1 of the Fused MoE paragraph.
+ *
+ *   logit[t,e] = sum_h x[t,h] * w[e,h],  x [T,H] and w [E,H] in bf16, result fp32.
+ *
+ * Indices selected from these logits are compared bit for bit, so the fp32
+ * summation order is part of the definition (H a multiple of 64):
+ *   - 32 partial sums p[0..31]; partial l takes the elements h with
+ *     (h / 2) mod 32 == l, i.e. the l-th pair of every run of 64 elements, in
+ *     increasing h: p[l] = fmaf(x[h], w[h], p[l]) (the product of two bf16
+ *     values is exact in fp32, so this is one rounding per element);
+ *   - then five pairwise rounds, d = 16, 8, 4, 2, 1: every p[l] becomes
+ *     p[l] + p[l xor d] (all l at once; fp32 addition is commutative, so both
+ *     partners get the same value); p[0] is the logit. */
+int moe_ref_router_logits(int T, int H, int E, const uint16_t *x_bf16,
+                          const uint16_t *w_bf16, float *logits)
+{
+    int t, e, h, l, d;
+    if (T < 0 || H <= 0 || E <= 0 || H % 64 != 0 || !logits || (T > 0 && (!x_bf16 || !w_bf16)))
+        return MOE_REF_BAD_ARG;
+    for (t = 0; t < T; ++t) {
+        for (e = 0; e < E; ++e) {
+            float p[32], q[32];
+            for (l = 0; l < 32; ++l)
+                p[l] = 0.0f;
+            for (h = 0; h < H; ++h) {
+                l = (h / 2) % 32;
+                p[l] = fmaf(moe_ref_bf16_decode(x_bf16[(size_t)t * H + h]),
+                            moe_ref_bf16_decode(w_bf16[(size_t)e * H + h]), p[l]);
+            }
+            for (d = 16; d >= 1; d /= 2) {
+                for (l = 0; l < 32; ++l)
+                    q[l] = p[l] + p[l ^ d];
+                for (l = 0; l < 32; ++l)
+                    p[l] = q[l];
+            }
+            logits[(size_t)t * E + e] = p[0];
+        }
+    }
+    return MOE_REF_OK;
+}
+
+/* Input-side quantisation of the activations as the workload description
+ * prescribes it (FP8 e4m3, one fp32 scale per token per 128 columns):
+ *   amax = max |x| over the block; scale = amax / 448 (1 if the block is all
+ *   zero); code = e4m3(x / scale), round to nearest even, saturating.
+ *   x [T,H] bf16 -> q [T,H] codes, scale [T,H/128]. */
+int moe_ref_quantize_rows(int T, int H, const uint16_t *x_bf16, uint8_t *q, float *scale)
+{
+    int t, b, i;
+    if (T < 0 || H <= 0 || H % QBLOCK != 0 || (T > 0 && (!x_bf16 || !q || !scale)))
+        return MOE_REF_BAD_ARG;
+    for (t = 0; t < T; ++t) {
+        for (b = 0; b < H / QBLOCK; ++b) {
+            const uint16_t *xb = x_bf16 + (size_t)t * H + (size_t)b * QBLOCK;
+            float amax = 0.0f, sc;
+            for (i = 0; i < QBLOCK; ++i) {
+                float a = fabsf(moe_ref_bf16_decode(xb[i]));
+                if (a > amax)
+                    amax = a;
+            }
+            sc = (amax == 0.0f) ? 1.0f : amax / 448.0f;
+            scale[(size_t)t * (H / QBLOCK) + b] = sc;
+            for (i = 0; i < QBLOCK; ++i)
+                q[(size_t)t * H + (size_t)b * QBLOCK + i] =
+                    moe_ref_e4m3_encode(moe_ref_bf16_decode(xb[i]) / sc);
+        }
+    }
+    return MOE_REF_OK;
 }
 
 /* Grouped routing of DeepSeek-V3 as the paper's stage 1 lists it (sigmoid,

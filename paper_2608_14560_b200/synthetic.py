@@ -146,6 +146,21 @@ def make_inputs(wl: Workload, device: str | torch.device = "cpu") -> dict:
     }
 
 
+def make_router_inputs(wl: Workload, device: str | torch.device = "cpu") -> dict:
+    """Inputs of the layer when it starts from hidden states: the bf16 hidden states whose quantisation
+    make_inputs returns as hidden_fp8 / hidden_scale (same generator, same first draw), and a router weight
+    [E, H] bf16 drawn N(0, 1/H) so that the logits have about unit variance."""
+    d = wl.dims
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(wl.seed)
+    hidden = torch.randn(wl.tokens, d.hidden, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    g2 = torch.Generator(device=dev)
+    g2.manual_seed(wl.seed + 500009)
+    w = torch.randn(d.num_experts, d.hidden, generator=g2, device=dev, dtype=torch.float32) / (d.hidden ** 0.5)
+    return {"hidden_bf16": hidden, "router_weight": w.to(torch.bfloat16)}
+
+
 def make_activations(wl: Workload, seed: int, device: str | torch.device = "cpu") -> dict:
     """A fresh set of per-step activations (hidden + logits) for the same layer,
     used to rotate inputs between timed iterations."""

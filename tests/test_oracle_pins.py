@@ -365,3 +365,104 @@ def test_forward_expert_parallel_shards_sum_to_all_local():
                      w2=inp["w2"][off:off + 4], w2_scale=inp["w2_scale"][off:off + 4], local_expert_offset=off)
         acc += oracle.bf16_decode(oracle.forward(shard, d.n_group, d.topk_group, d.top_k)["out"])
     assert np.abs(acc - full).max() <= 4 * 2.0 ** -8 * np.abs(full).max()
+
+
+# --------------------------------------------------------------------------
+# router projection and input quantisation (the layer started from bf16 hidden states)
+# --------------------------------------------------------------------------
+def _bf16_bits(x):
+    return torch.as_tensor(np.asarray(x, np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+def test_router_projection_hand_worked_cases():
+    def vec(spec, ramp_ok=True):
+        v = np.zeros(64, np.float32)
+        spec = spec.strip()
+        if spec == "ramp":
+            return np.arange(1, 65, dtype=np.float32)
+        if spec == "ones":
+            return np.ones(64, np.float32)
+        if spec == "alt":
+            return np.where(np.arange(64) % 2 == 0, 1.0, -1.0).astype(np.float32)
+        for item in spec.split():
+            k, val = item.split(":")
+            if k == "even":
+                v[0::2] = float(val)
+            else:
+                v[int(k)] = float(val)
+        return v
+
+    n = 0
+    for line in open(os.path.join(GOLDEN, "router_projection.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        _, xs, ws, want = [f.strip() for f in line.split("|")]
+        x = vec(xs)[None, :]
+        w = np.stack([vec(f) for f in ws.split(";")])
+        got = oracle.router_logits(_bf16_bits(x), _bf16_bits(w))
+        assert got.shape == (1, w.shape[0])
+        assert got[0].tolist() == [float(v) for v in want.split()], line
+        n += 1
+    assert n == 2
+
+
+@pytest.mark.parametrize("T,H,E,seed", [(5, 64, 7, 0), (9, 448, 16, 1), (3, 7168, 256, 2)])
+def test_router_projection_vs_fp64_library_matmul(T, H, E, seed):
+    rng = np.random.default_rng(seed)
+    x = _bf16_bits(rng.standard_normal((T, H)))
+    w = _bf16_bits(rng.standard_normal((E, H)) / np.sqrt(H))
+    got = oracle.router_logits(x, w).astype(np.float64)
+    xd = torch.from_numpy(oracle.bf16_decode(x).astype(np.float64))
+    wd = torch.from_numpy(oracle.bf16_decode(w).astype(np.float64))
+    ref = torch.matmul(xd, wd.t()).numpy()
+    # fp32 summation: each of the (H/32 + 5) roundings on the path of a term is at most half an ulp of a
+    # running value bounded by the sum of magnitudes
+    bound = (H / 32 + 6) * 2.0 ** -24 * torch.matmul(xd.abs(), wd.abs().t()).numpy()
+    assert (np.abs(got - ref) <= bound).all()
+    # a transposed or mis-strided operand would fail by orders of magnitude; so would a dropped pair
+    assert np.abs(got - ref).max() < 1e-4
+
+
+def test_router_projection_rows_and_experts_are_independent():
+    rng = np.random.default_rng(3)
+    x = _bf16_bits(rng.standard_normal((6, 128)))
+    w = _bf16_bits(rng.standard_normal((10, 128)))
+    full = oracle.router_logits(x, w)
+    assert np.array_equal(oracle.router_logits(x[2:5], w[3:9]), full[2:5, 3:9])
+    # doubling a weight row doubles its logits bit for bit (powers of two commute with rounding)
+    w2 = _bf16_bits(2.0 * oracle.bf16_decode(w))
+    assert np.array_equal(oracle.router_logits(x, w2), 2.0 * full)
+
+
+def test_input_quantisation_vs_torch_cast():
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((7, 512)).astype(np.float32) * rng.choice([1e-3, 0.3, 1.0, 40.0], (7, 1)).astype(np.float32)
+    x[1, 128:256] = 0.0            # an all-zero block: scale 1, codes 0
+    x[2, 5] = 448.0                # values at the format's edge
+    xb = torch.from_numpy(x).to(torch.bfloat16)
+    q, s = oracle.quantize_rows(xb.view(torch.int16).numpy().view(np.uint16))
+    xf = xb.to(torch.float32).view(7, 4, 128)
+    amax = xf.abs().amax(-1)
+    ts = torch.where(amax == 0, torch.ones_like(amax), amax / 448.0)
+    tq = (xf / ts.unsqueeze(-1)).to(torch.float8_e4m3fn).view(7, 512).view(torch.uint8).numpy()
+    assert np.array_equal(s.view(np.uint32), ts.numpy().view(np.uint32))
+    assert np.array_equal(q, tq)
+    assert s[1, 1] == 1.0 and not q[1, 128:256].any()
+    # the synthetic input recipe applies the same rule
+    rq, rs = syn._quant_rows_128(xb.to(torch.float32))
+    assert np.array_equal(q, rq.view(torch.uint8).numpy()) and np.array_equal(s, rs.numpy())
+
+
+def test_forward_from_hidden_is_projection_then_quantisation_then_forward():
+    wl = syn.tiny_workload(tokens=6, hidden=256, intermediate=128)
+    inp = syn.to_host(syn.make_inputs(wl))
+    r = syn.to_host(syn.make_router_inputs(wl))
+    d = wl.dims
+    res = oracle.forward_from_hidden({**inp, **r}, d.n_group, d.topk_group, d.top_k)
+    logits = oracle.router_logits(r["hidden_bf16"], r["router_weight"])
+    q, s = oracle.quantize_rows(r["hidden_bf16"])
+    direct = oracle.forward(dict(inp, hidden_fp8=q, hidden_scale=s, router_logits=logits), d.n_group, d.topk_group,
+                            d.top_k)
+    assert np.array_equal(res["out"], direct["out"]) and np.array_equal(res["topk_idx"], direct["topk_idx"])
+    # the recipe's own FP8 activations are the quantisation of the same bf16 hidden states
+    assert np.array_equal(q, inp["hidden_fp8"]) and np.array_equal(s, inp["hidden_scale"])
