@@ -112,6 +112,33 @@ int moe_fp8_forward_host(moe_fp8_handle_t h, int T, const void* host_hidden_fp8,
                          float scaling_factor, void* host_out, void* stream);
 
 /*
+ * The same pass started from bf16 hidden states: stage 1 of the Fused MoE description begins with "routing
+ * scores via a lightweight linear projection", and the FP8 activations with their 128-wide scales are the
+ * quantisation of those hidden states.  This entry computes
+ *   router_logits[t, e] = sum_h hidden[t, h] * router_weight[e, h]        (bf16 inputs, fp32 result)
+ *   hidden_fp8, hidden_scale = per token per 128 columns: scale = amax / 448 (1 for an all-zero block),
+ *                              code = e4m3(x / scale), round to nearest even, saturating
+ * into staging areas of the workspace and then runs moe_fp8_forward on them (two more kernel launches).
+ * Because the selected expert indices are reproducible bit for bit, the fp32 summation order of the
+ * projection is fixed: 32 partial sums, partial l takes the l-th pair of every run of 64 elements in
+ * increasing order with one fused multiply-add per element, then five pairwise rounds p[l] += p[l xor d],
+ * d = 16, 8, 4, 2, 1.
+ *
+ *   hidden_bf16    bf16 [T, H]     device
+ *   router_weight  bf16 [256, H]   device
+ * All other arguments as moe_fp8_forward.  The staging areas are shared with moe_fp8_forward_host.
+ */
+int moe_fp8_forward_from_hidden(moe_fp8_handle_t h, int T, const void* hidden_bf16, const void* router_weight,
+                                const void* routing_bias, const void* w13, const float* w13_scale, const void* w2,
+                                const float* w2_scale, int local_expert_offset, float scaling_factor, void* out,
+                                void* stream);
+/* Test hook: copies what the last moe_fp8_forward_from_hidden (or moe_fp8_forward_host) on this handle fed
+ * to the forward pass -- router_logits fp32 [T,256], hidden_fp8 e4m3 [T,H], hidden_scale fp32 in the
+ * configured layout -- into caller buffers (device pointers, any may be NULL), enqueued on `stream`. */
+int moe_fp8_debug_export_inputs(moe_fp8_handle_t h, int T, float* router_logits, void* hidden_fp8,
+                                float* hidden_scale, void* stream);
+
+/*
  * Test hook: copies internal results of the LAST forward on this handle into
  * caller buffers (device pointers, any may be NULL), enqueued on `stream`.
  *   topk_idx       int32 [T, 8]  selected experts, descending biased score

@@ -18,7 +18,7 @@ EXPORTS = (
     "moe_fp8_forward_host", "moe_fp8_debug_export", "moe_fp8_last_cuda_error", "moe_fp8_last_launch_count",
     "moe_fp8_strerror", "moe_fp8_set_stage_timing", "moe_fp8_num_stages", "moe_fp8_stage_name",
     "moe_fp8_get_stage_times", "moe_fp8_expert_histogram_static", "moe_fp8_debug_set_fault",
-    "moe_fp8_debug_sigmoid",
+    "moe_fp8_debug_sigmoid", "moe_fp8_forward_from_hidden", "moe_fp8_debug_export_inputs",
 )
 
 
@@ -59,6 +59,10 @@ def load_library() -> C.CDLL:
         lib.moe_fp8_forward.restype = C.c_int
         lib.moe_fp8_forward_host.argtypes = fwd
         lib.moe_fp8_forward_host.restype = C.c_int
+        lib.moe_fp8_forward_from_hidden.argtypes = [vp, C.c_int, vp, vp, vp, vp, fp, vp, fp, C.c_int, C.c_float, vp, vp]
+        lib.moe_fp8_forward_from_hidden.restype = C.c_int
+        lib.moe_fp8_debug_export_inputs.argtypes = [vp, C.c_int, fp, vp, fp, vp]
+        lib.moe_fp8_debug_export_inputs.restype = C.c_int
         lib.moe_fp8_debug_export.argtypes = [vp, C.c_int, ip, fp, ip, ip, ip, vp, fp, vp, ip, vp]
         lib.moe_fp8_debug_export.restype = C.c_int
         lib.moe_fp8_last_cuda_error.argtypes = [vp]
@@ -181,6 +185,29 @@ class MoeFp8:
             _ptr(inp["w2_scale"]), int(inp["local_expert_offset"]), float(inp["scaling_factor"]), _ptr(out),
             self._stream(stream)))
         return out
+
+    def forward_from_hidden(self, inp: dict, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+        """moe_fp8_forward_from_hidden: inp carries hidden_bf16 [T,H] and router_weight [256,H] (bf16) besides
+        the bias and the expert weights."""
+        T = inp["hidden_bf16"].shape[0]
+        if out is None:
+            out = torch.empty(T, self.cfg.hidden, dtype=torch.bfloat16, device=self.device)
+        self._check(self.lib.moe_fp8_forward_from_hidden(
+            self.handle, T, _ptr(inp["hidden_bf16"]), _ptr(inp["router_weight"]), _ptr(inp["routing_bias"]),
+            _ptr(inp["w13"]), _ptr(inp["w13_scale"]), _ptr(inp["w2"]), _ptr(inp["w2_scale"]),
+            int(inp["local_expert_offset"]), float(inp["scaling_factor"]), _ptr(out), self._stream(stream)))
+        return out
+
+    def debug_export_inputs(self, T: int, stream=None) -> dict:
+        """moe_fp8_debug_export_inputs -> router_logits, hidden_fp8 (uint8 codes), hidden_scale (device tensors)."""
+        dev, H = self.device, self.cfg.hidden
+        sshape = (H // 128, T) if self.cfg.hidden_scale_layout else (T, H // 128)
+        r = {"router_logits": torch.empty(T, self.cfg.num_experts, dtype=torch.float32, device=dev),
+             "hidden_fp8": torch.empty(T, H, dtype=torch.uint8, device=dev),
+             "hidden_scale": torch.empty(sshape, dtype=torch.float32, device=dev)}
+        self._check(self.lib.moe_fp8_debug_export_inputs(self.handle, T, _ptr(r["router_logits"]), _ptr(r["hidden_fp8"]),
+                                                         _ptr(r["hidden_scale"]), self._stream(stream)))
+        return r
 
     def forward_host(self, host_act: dict, weights: dict, host_out: torch.Tensor, stream=None) -> torch.Tensor:
         """moe_fp8_forward_host: hidden_fp8 / hidden_scale / router_logits / out in (pinned) host memory."""

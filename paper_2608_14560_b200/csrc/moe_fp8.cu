@@ -15,6 +15,7 @@
 #include "permute.cuh"
 #include "gemm.cuh"
 #include "combine.cuh"
+#include "router.cuh"
 
 namespace {
 
@@ -236,6 +237,9 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     e = cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
     if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
     e = cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
+    e = cudaFuncSetAttribute(router_logits_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(router_smem_bytes(4, 4)));
     if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
     e = cudaFuncSetAttribute(route_permute_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(route_permute_smem_bytes(P_TAIL_MAX_TOKENS, P_MAX_LOCAL)));
@@ -529,6 +533,60 @@ int moe_fp8_forward_host(moe_fp8_handle_t h, int T, const void* host_hidden_fp8,
     if ((e = cudaMemcpyAsync(host_out, d_out, Tz * H * 2, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
         return cuda_fail(h, e);
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(h, e);
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_forward_from_hidden(moe_fp8_handle_t h, int T, const void* hidden_bf16, const void* router_weight,
+                                const void* routing_bias, const void* w13, const float* w13_scale, const void* w2,
+                                const float* w2_scale, int local_expert_offset, float scaling_factor, void* out,
+                                void* stream_v) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    if (T < 0 || T > h->cfg.max_tokens) return MOE_FP8_ERR_BAD_ARG;
+    if (!router_weight || misaligned(router_weight) || (T > 0 && (!hidden_bf16 || misaligned(hidden_bf16))))
+        return MOE_FP8_ERR_BAD_ARG;
+    if (!h->ws) return MOE_FP8_ERR_NO_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int H = h->cfg.hidden, E = h->cfg.num_experts;
+    uint8_t* d_hidden = at<uint8_t>(h, h->L.stage_hidden);
+    float* d_scale = at<float>(h, h->L.stage_scale);
+    float* d_logits = at<float>(h, h->L.stage_logits);
+    if (T > 0) {
+        const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(hidden_bf16);
+        const __nv_bfloat16* wr = static_cast<const __nv_bfloat16*>(router_weight);
+        cudaError_t e;
+        if (T <= 128)  // few tokens: many small CTAs, so that the router weight streams in from many SMs
+            e = launch(router_logits_kernel<1, 4>, dim3((T + 7) / 8, E / 32), 128, router_smem_bytes(1, 4), stream, false,
+                       T, H, E, x, wr, d_logits);
+        else
+            e = launch(router_logits_kernel<4, 4>, dim3((T + 31) / 32, E / 32), 512, router_smem_bytes(4, 4), stream,
+                       false, T, H, E, x, wr, d_logits);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+        const long long blocks = (static_cast<long long>(T) * (H / 128) + 7) / 8;
+        e = launch(quantize_rows_kernel, static_cast<int>(std::min<long long>(blocks, h->sm_count * 16LL)), 256, 0, stream,
+                   false, T, H, h->cfg.hidden_scale_layout, x, d_hidden, d_scale);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    const int rc = moe_fp8_forward(h, T, d_hidden, d_scale, d_logits, routing_bias, w13, w13_scale, w2, w2_scale,
+                                   local_expert_offset, scaling_factor, out, stream_v);
+    if (rc == MOE_FP8_OK && T > 0) h->last_launches += 2;
+    return rc;
+}
+
+int moe_fp8_debug_export_inputs(moe_fp8_handle_t h, int T, float* router_logits, void* hidden_fp8,
+                                float* hidden_scale, void* stream_v) {
+    if (!h || T < 0 || T > h->cfg.max_tokens) return MOE_FP8_ERR_BAD_ARG;
+    if (!h->ws) return MOE_FP8_ERR_NO_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const size_t Tz = T, H = h->cfg.hidden;
+    cudaError_t e = cudaSuccess;
+    auto copy = [&](void* dst, size_t off, size_t bytes) {
+        if (dst && bytes && e == cudaSuccess)
+            e = cudaMemcpyAsync(dst, h->ws + off, bytes, cudaMemcpyDeviceToDevice, stream);
+    };
+    copy(router_logits, h->L.stage_logits, Tz * h->cfg.num_experts * 4);
+    copy(hidden_fp8, h->L.stage_hidden, Tz * H);
+    copy(hidden_scale, h->L.stage_scale, Tz * (H / 128) * 4);
+    if (e != cudaSuccess) return cuda_fail(h, e);
     return MOE_FP8_OK;
 }
 

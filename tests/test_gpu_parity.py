@@ -271,3 +271,54 @@ def test_a_wait_that_runs_out_is_reported_and_the_handle_stays_usable(cuda_devic
     assert torch.equal(got.view(torch.int16), want.view(torch.int16))
     run_and_compare(wl, cuda_device, inp=inp, eng=eng)
     eng.close()
+
+
+# ---- the layer started from bf16 hidden states (router projection + input quantisation in front) ----------
+def _from_hidden_case(wl, device, sample_tokens=None, **kw):
+    d = wl.dims
+    inp = syn.make_inputs(wl, device)
+    r = syn.make_router_inputs(wl, device)
+    eng = make_engine(wl, device, **kw)
+    out = eng.forward_from_hidden({**inp, **r})
+    fed = eng.debug_export_inputs(wl.tokens)
+    dbg = eng.debug_export(wl.tokens, rows=False)
+    torch.cuda.synchronize()
+    assert int(dbg["status"].item()) == 0
+    host = syn.to_host({**inp, **r})
+    # projection and quantisation: bit for bit (the summation order of the projection is part of its definition)
+    logits = oracle.router_logits(host["hidden_bf16"], host["router_weight"])
+    assert np.array_equal(fed["router_logits"].cpu().numpy().view(np.uint32), logits.view(np.uint32)), \
+        "router logits differ from the oracle's fixed-order sum"
+    q, s = oracle.quantize_rows(host["hidden_bf16"])
+    assert np.array_equal(fed["hidden_fp8"].cpu().numpy(), q)
+    gs = fed["hidden_scale"].cpu().numpy()
+    assert np.array_equal(gs.T if eng.cfg.hidden_scale_layout else gs, s)
+    # routing from those logits: indices and weights bit for bit
+    ridx, rw = oracle.route(logits, host["routing_bias"], d.n_group, d.topk_group, d.top_k, float(inp["scaling_factor"]))
+    assert np.array_equal(dbg["topk_idx"].cpu().numpy(), ridx)
+    assert np.array_equal(dbg["topk_w"].cpu().numpy(), rw)
+    # output
+    tokens = np.arange(wl.tokens, dtype=np.int32) if sample_tokens is None else sample_tokens
+    full = dict(host, hidden_fp8=q, hidden_scale=s, router_logits=logits)
+    from parity import oracle_forward_parallel
+    ref = oracle_forward_parallel(full, d, tokens)
+    gpu = out.view(torch.int16).cpu().numpy().view(np.uint16)[tokens]
+    check_output(gpu, ref)
+    eng.close()
+    return int(((ridx >= wl.local_expert_offset) & (ridx < wl.local_expert_offset + d.num_local_experts)).sum())
+
+
+@pytest.mark.parametrize("tokens", [1, 8, 33, 128, 129, 700])  # 128 | 129: the two projection tile shapes
+def test_from_hidden_small_layer(cuda_device, tokens):
+    _from_hidden_case(_wl(tokens, seed=60 + tokens), cuda_device)
+
+
+def test_from_hidden_transposed_scale_layout(cuda_device):
+    _from_hidden_case(_wl(77, seed=59), cuda_device, hidden_scale_layout=1)
+
+
+@pytest.mark.parametrize("cfg,n_sample", [(1, 64), (2, 128)])
+def test_from_hidden_benchmark_shapes(cuda_device, cfg, n_sample):
+    wl = syn.CONFIGS[cfg]
+    S = _from_hidden_case(wl, cuda_device, sample_tokens=_sample(wl.tokens, n_sample, cfg))
+    assert S > 0
