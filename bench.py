@@ -45,6 +45,7 @@ HBM_DATASHEET_GBS = 8000.0
 NCU_TRAFFIC_RATIO = {
     ("hbm", "gemm1_swiglu_quant"): 1.035, ("hbm", "gemm2"): 1.02,
     ("tensor", "gemm1_swiglu_quant"): 1.14, ("tensor", "gemm2"): 1.10,
+    ("hbm", "fused_small"): 1.03,
 }
 METRIC = "fused FP8 MoE forward throughput (tokens/s; TFLOPS and roofline fraction alongside)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -277,9 +278,11 @@ def run_cuda_config(wl, device, steps, warmup, peaks, peak_kind, want_e2e=True, 
     dom_s = stage_avg[dom] * 1e-3
     g1_flops = 2 * d.hidden * 2 * d.intermediate * S
     g2_flops = 2 * d.intermediate * d.hidden * S
-    kern_flops = {"gemm1_swiglu_quant": g1_flops, "gemm2": g2_flops}.get(dom, 0.0)
-    kern_bytes = {"gemm1_swiglu_quant": W13_BYTES_PER_EXPERT * A + S * (d.hidden + d.hidden // 32 + d.intermediate),
-                  "gemm2": W2_BYTES_PER_EXPERT * A + S * (d.intermediate + 2 * d.hidden)}.get(dom, 0.0)
+    kern_flops = {"gemm1_swiglu_quant": g1_flops, "gemm2": g2_flops, "fused_small": g1_flops + g2_flops}.get(dom, 0.0)
+    b1 = W13_BYTES_PER_EXPERT * A + S * (d.hidden + d.hidden // 32 + d.intermediate)
+    b2 = W2_BYTES_PER_EXPERT * A + S * (d.intermediate + 2 * d.hidden)
+    # (the single kernel of a small batch reads both weight sets, the token rows, and writes the output)
+    kern_bytes = {"gemm1_swiglu_quant": b1, "gemm2": b2, "fused_small": b1 + b2 + T * d.hidden * 2}.get(dom, 0.0)
     fp8_peak = 2.0 * peaks["bf16_tflops_sustained" if ms * steps > 500 else "bf16_tflops"]
     if kern_flops / (fp8_peak * 1e12) > kern_bytes / (peaks["hbm_gbs"] * 1e9):
         ach = kern_flops / dom_s / 1e12

@@ -157,13 +157,22 @@ int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w
                          int* status_word, void* stream);
 
 /*
+ * Batches of at most 32 tokens run the gather of stage 2, both GEMMs of stage 3 and the combine of stage 4 as
+ * ONE kernel behind the routing kernel (the paper's short regime, T = 1-16, is bounded by routing and launch
+ * overhead, and it names fusing the scatter into GEMM2's epilogue as the next step; in that kernel the CTA that
+ * stores the last local row of a token sums the token's rows in routing order, so results stay bit-identical
+ * to the separate kernels).  On by default; enable = 0 makes such batches take the separate kernels too.
+ */
+int moe_fp8_set_small_batch_fusion(moe_fp8_handle_t h, int enable);
+
+/*
  * Test hook for the failure path of the bounded device waits (every wait on an mbarrier inside the GEMM
  * kernels gives up after a limit, records a fault code in the status word and lets the kernel return with
  * its tensor memory released).  skip_iteration >= 0: in the next forwards the copy producer of every CTA
  * of the GEMM1 kernel stops before its skip_iteration-th pipeline stage, so the consumers wait for a stage
  * that nothing fills; wait_clocks > 0 shortens the limit of every wait to that many SM clocks (0 restores
  * the default of about a second).  skip_iteration < 0 switches the hook off.  Nothing traps: the forward
- * returns normally, its output is garbage and the status word holds a time-out code (1..5).
+ * returns normally, its output is garbage and the status word holds a time-out code (1..5, 8).
  */
 int moe_fp8_debug_set_fault(moe_fp8_handle_t h, int skip_iteration, long long wait_clocks);
 

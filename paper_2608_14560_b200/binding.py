@@ -19,6 +19,7 @@ EXPORTS = (
     "moe_fp8_strerror", "moe_fp8_set_stage_timing", "moe_fp8_num_stages", "moe_fp8_stage_name",
     "moe_fp8_get_stage_times", "moe_fp8_expert_histogram_static", "moe_fp8_debug_set_fault",
     "moe_fp8_debug_sigmoid", "moe_fp8_forward_from_hidden", "moe_fp8_debug_export_inputs",
+    "moe_fp8_set_small_batch_fusion",
 )
 
 
@@ -79,6 +80,8 @@ def load_library() -> C.CDLL:
         lib.moe_fp8_get_stage_times.restype = C.c_int
         lib.moe_fp8_expert_histogram_static.argtypes = [C.c_int, ip, C.c_int, C.c_int, ip, ip, vp]
         lib.moe_fp8_expert_histogram_static.restype = C.c_int
+        lib.moe_fp8_set_small_batch_fusion.argtypes = [vp, C.c_int]
+        lib.moe_fp8_set_small_batch_fusion.restype = C.c_int
         lib.moe_fp8_debug_set_fault.argtypes = [vp, C.c_int, C.c_longlong]
         lib.moe_fp8_debug_set_fault.restype = C.c_int
         lib.moe_fp8_debug_sigmoid.argtypes = [C.c_int, fp, fp, vp]
@@ -219,6 +222,10 @@ class MoeFp8:
             int(weights["local_expert_offset"]), float(weights["scaling_factor"]), _ptr(host_out),
             self._stream(stream)))
         return host_out
+
+    def set_small_batch_fusion(self, enable: bool):
+        """moe_fp8_set_small_batch_fusion: batches of <= 32 tokens as one fused kernel (default) or as separate ones."""
+        self._check(self.lib.moe_fp8_set_small_batch_fusion(self.handle, int(enable)))
 
     def debug_set_fault(self, skip_iteration: int = -1, wait_clocks: int = 0):
         """moe_fp8_debug_set_fault (test hook of the bounded-wait failure path)."""

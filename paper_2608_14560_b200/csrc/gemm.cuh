@@ -22,6 +22,18 @@
 //               tile apply the fused tail and store.
 // Scales are arbitrary fp32 (amax/448), so the power-of-two hardware block
 // scaling cannot express them; the per-K-block promotion is done on the ALUs.
+//
+// Two kernels are built from these roles:
+//   grouped_gemm_kernel<MODE>   one GEMM per launch (any batch size);
+//   fused_small_kernel          batches of at most F_MAX_TOKENS tokens: the gather of stage 2, GEMM1, GEMM2
+//               and the weighted combine of stage 4 in ONE launch.  Every CTA first works through its GEMM1
+//               tiles, then its GEMM2 tiles.  Warp 3 gathers the (few) token rows of a GEMM1 tile straight
+//               from the token-major input with cp.async.  A GEMM2 tile starts once a counter in global
+//               memory says that all GEMM1 column tiles of its row tile have been stored (bounded wait; GEMM1
+//               tiles never wait for another CTA and precede the GEMM2 tiles in every CTA, and all CTAs of
+//               the one-per-SM grid are resident, so the counter always arrives).  The CTA that completes the
+//               last local row of a token for a column tile -- found with a per-(token, column tile)
+//               counter, nobody waits -- sums that token's rows in routing order and writes the bf16 output.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
@@ -30,30 +42,49 @@
 
 namespace moe {
 
-constexpr int G_STAGES = 4;
+
+
 // The two MMA issuer threads take the even and the odd K-blocks.  A thread must see EVERY phase of a barrier it
 // waits on (a parity wait cannot tell the wanted phase from the one two earlier), so a stage must always fall
-// to the same issuer: the stage count has to be even.
-static_assert(G_STAGES % 2 == 0, "an odd stage count lets an issuer thread skip phases of full[s]");
+// to the same issuer: the stage count has to be even (checked in Geometry).
+constexpr int G_MAX_STAGES = 6;
 constexpr int G_BLOCK_K = 128;                          // K bytes per stage = one scale block
 constexpr int G_TILE_N = 256;                           // output columns per tile
 constexpr int G_HALF_N = 128;                           // columns handled by one epilogue warpgroup
 constexpr int G_ACC_BUFS = 2;                           // TMEM accumulator buffers (2 x 256 columns)
-constexpr int G_A_BYTES = TILE_M * G_BLOCK_K;           // 16 KB
 constexpr int G_B_BYTES = G_TILE_N * G_BLOCK_K;         // 32 KB
-constexpr int G_STAGE_BYTES = G_A_BYTES + G_B_BYTES;    // 48 KB
-constexpr int G_SCALE_RING = 8;                         // K-blocks of activation scales in flight
-constexpr int G_SCALE_BYTES = TILE_M * 4;               // 512 B per K-block
 constexpr int G_THREADS = 384;                          // 4 control warps + 8 epilogue warps
 constexpr int G_EPI_WARPS = 8;
 constexpr int G_STORE_WARP_BYTES = 2048;                // per-warp staging: 32 rows x 64 B (swizzled)
-constexpr int G_STORE_BYTES = G_EPI_WARPS * G_STORE_WARP_BYTES;
 constexpr int G_AMAX_BYTES = 2 * 2 * TILE_M * 4;               // GEMM1 row-amax exchange
 constexpr int G_CTRL_BYTES = 512;
-constexpr int G_SMEM_BYTES = G_STAGES * G_STAGE_BYTES + G_SCALE_RING * G_SCALE_BYTES + G_STORE_BYTES +
-                             G_AMAX_BYTES + G_CTRL_BYTES + 1024;       // + alignment slack
 constexpr uint32_t G_TMEM_COLS = 512;
-static_assert(G_SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+
+// Shared-memory geometry of a kernel: pipeline stages, rows of the A tile that are actually fetched (the MMA
+// always reads 128 rows; with fewer fetched rows the rest of its A operand is whatever follows in shared
+// memory, and those accumulator rows are never stored), slots of the activation-scale ring.
+template <int STAGES_, int A_ROWS_, int SCALE_SLOTS_, int STORE_BYTES_>
+struct Geometry {
+    static constexpr int STAGES = STAGES_, A_ROWS = A_ROWS_, SCALE_SLOTS = SCALE_SLOTS_;
+    static constexpr int A_BYTES = A_ROWS_ * G_BLOCK_K;
+    static constexpr int STAGE_BYTES = A_BYTES + G_B_BYTES;
+    static constexpr int SCALE_BYTES = A_ROWS_ * 4;                  // per K-block
+    static constexpr int STORE_BYTES = STORE_BYTES_;                 // GEMM1 output staging
+    static constexpr int SMEM_BYTES = STAGES_ * STAGE_BYTES + SCALE_SLOTS_ * SCALE_BYTES + STORE_BYTES_ + G_AMAX_BYTES +
+                                      G_CTRL_BYTES + 1024;           // + alignment slack
+    static_assert(STAGES_ % 2 == 0, "an odd stage count lets an issuer thread skip phases of full[s]");
+    static_assert(STAGES_ <= G_MAX_STAGES, "control block holds G_MAX_STAGES barriers per kind");
+    static_assert(A_BYTES % 1024 == 0, "the B tile must stay 1024-byte aligned for the 128-byte swizzle");
+    static_assert(SCALE_SLOTS_ >= STAGES_ + G_ACC_BUFS + 1, "the producer may be that far ahead of the epilogue");
+    static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA may use");
+};
+// one GEMM per launch: full 128-row A tiles, 4 stages of 48 KB
+using GeomFull = Geometry<4, TILE_M, 8, G_EPI_WARPS * G_STORE_WARP_BYTES>;
+// fused small-batch kernel: a row tile holds at most 32 rows, so the A slot shrinks to 4 KB and six stages fit:
+// 192 KB of weights in flight per SM instead of 128 KB, which is what a weight-streaming CTA is limited by
+using GeomSmall = Geometry<6, 32, 16, 2 * G_STORE_WARP_BYTES>;
+
+constexpr int F_MAX_TOKENS = GeomSmall::A_ROWS;   // largest batch of fused_small_kernel
 
 struct GemmArgs {
     int num_kb;               // K / 128
@@ -75,12 +106,27 @@ struct GemmArgs {
     int fault_skip_it;        // test hook: the producer stops before this pipeline iteration (-1: never)
 };
 
+// What fused_small_kernel needs beyond the two GemmArgs.
+struct FusedArgs {
+    int T, H, scale_layout;
+    const uint8_t* hidden;        // e4m3 [T, H] token-major activations
+    const float* hidden_scale;    // [T, H/128] or [H/128, T]
+    const int* row_token;         // padded row -> token
+    const int* slot_to_row;       // [T*8]
+    const float* topk_w;          // [T*8]
+    const int* tok_nlocal;        // [T] local slots of each token
+    int* ready;                   // [row tiles] GEMM1 column tiles stored, zero at launch
+    int* tok_done;                // [T, H/256] GEMM2 rows stored per (token, column tile), zero at launch
+    __nv_bfloat16* out;           // bf16 [T, H]
+};
+
 struct GemmCtrl {
-    uint64_t full[G_STAGES];   // stage filled (TMA transaction bytes)
-    uint64_t done[G_STAGES];   // the MMAs that read the stage have finished: stage free AND accumulator ready
+    uint64_t full[G_MAX_STAGES];   // stage filled (TMA transaction bytes)
+    uint64_t done[G_MAX_STAGES];   // the MMAs that read the stage have finished: stage free AND accumulator ready
     uint64_t tmem_empty[G_ACC_BUFS];
     uint64_t amax_bar[2];
     uint64_t drain_bar[2];
+    uint64_t sync_bar[2];      // fused kernel: rendezvous of the epilogue warps at the end of a tile
     uint32_t tmem_slot;
     int abort_flag;
 };
@@ -91,26 +137,46 @@ __device__ __forceinline__ void raise(GemmCtrl* c, int* status, int code) {
     atomicCAS(status, DEV_OK, code);
 }
 
-// MODE 1: gate/up projection + SwiGLU + re-quantisation (B tile = 4 x 64 weight rows:
-//         gate[0,64) | up[0,64) | gate[64,128) | up[64,128) of the tile's 128 columns).
-//         tmOut describes the e4m3 output [row_cap, I] for 64-byte x 32-row TMA stores.
-// MODE 2: down projection, bf16 rows out in the tile-blocked layout (B tile = 2 x 128 rows).
-template <int MODE>
-__global__ void __launch_bounds__(G_THREADS, 1)
-grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const __grid_constant__ CUtensorMap tmOut, const GemmArgs g) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    float* scale_ring = reinterpret_cast<float*>(smem + G_STAGES * G_STAGE_BYTES);
-    uint8_t* store_stage = smem + G_STAGES * G_STAGE_BYTES + G_SCALE_RING * G_SCALE_BYTES;
-    GemmCtrl* ctrl = reinterpret_cast<GemmCtrl*>(store_stage + G_STORE_BYTES + G_AMAX_BYTES);
-    volatile int* abort_flag = &ctrl->abort_flag;
-    const uint32_t smem_base = smem_u32(smem);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+// Byte offset of the 32-byte group holding columns [16*c16, 16*c16+16) of padded row r in the
+// tile-blocked bf16 output of GEMM2 (n_tiles = H / 256 column tiles).
+__host__ __device__ __forceinline__ size_t y_block_offset(int r, int c16, int n_tiles) {
+    const int m_tile = r / TILE_M, quad = (r % TILE_M) / 32, lane = r % 32;
+    const int n = c16 / 16, half = (c16 % 16) / 8, q = c16 % 8;
+    return (((static_cast<size_t>(m_tile) * n_tiles + n) * 2 + half) * 4 + quad) * 8192 + q * 1024 + lane * 32;
+}
 
+// The CTA's carve-up of shared memory and the values every role needs.
+struct Cta {
+    float* scale_ring;
+    uint8_t* store_stage;
+    float* amax_x;             // [2][2][TILE_M] GEMM1 row-amax exchange
+    GemmCtrl* ctrl;
+    volatile int* abort_flag;
+    uint32_t smem_base, tmem_base;
+    long long limit;
+    int warp, lane;
+};
+
+// Tiles first, first + stride, ... below count.
+struct TileRange {
+    int first, count, stride;
+};
+
+template <class GEO>
+__device__ __forceinline__ void gemm_cta_setup(Cta& c, uint8_t* smem_raw, int full_count) {
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    c.scale_ring = reinterpret_cast<float*>(smem + GEO::STAGES * GEO::STAGE_BYTES);
+    c.store_stage = smem + GEO::STAGES * GEO::STAGE_BYTES + GEO::SCALE_SLOTS * GEO::SCALE_BYTES;
+    c.amax_x = reinterpret_cast<float*>(c.store_stage + GEO::STORE_BYTES);
+    c.ctrl = reinterpret_cast<GemmCtrl*>(c.store_stage + GEO::STORE_BYTES + G_AMAX_BYTES);
+    c.abort_flag = &c.ctrl->abort_flag;
+    c.smem_base = smem_u32(smem);
+    c.warp = threadIdx.x >> 5;
+    c.lane = threadIdx.x & 31;
+    GemmCtrl* ctrl = c.ctrl;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < G_STAGES; ++s) {
-            mbar_init(smem_u32(&ctrl->full[s]), 1);
+        for (int s = 0; s < GEO::STAGES; ++s) {
+            mbar_init(smem_u32(&ctrl->full[s]), full_count);
             mbar_init(smem_u32(&ctrl->done[s]), 1);
         }
         for (int b = 0; b < G_ACC_BUFS; ++b) {
@@ -120,14 +186,480 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         mbar_init(smem_u32(&ctrl->amax_bar[1]), G_EPI_WARPS * 32);
         mbar_init(smem_u32(&ctrl->drain_bar[0]), 1);
         mbar_init(smem_u32(&ctrl->drain_bar[1]), 1);
+        mbar_init(smem_u32(&ctrl->sync_bar[0]), G_EPI_WARPS * 32);
+        mbar_init(smem_u32(&ctrl->sync_bar[1]), G_EPI_WARPS * 32);
         ctrl->abort_flag = 0;
         mbar_fence_init();
     }
-    if (warp == 1) {
+    if (c.warp == 1) {
         tmem_alloc(smem_u32(&ctrl->tmem_slot), G_TMEM_COLS);
         tmem_relinquish();
     }
-    if (warp == 0 && lane == 0) {
+}
+
+// ---------------- TMA producer (one thread) ----------------
+// MODE 1: B tile = 4 x 64 weight rows (gate[0,64) | up[0,64) | gate[64,128) | up[64,128) of the tile's 128
+// columns); MODE 2: B tile = 2 x 128 rows.  FUSED and MODE 1: the A tile and the scales come from the gather
+// warp instead; FUSED and MODE 2: the tile's A rows are GEMM1's output and must have been stored.
+template <int MODE, bool FUSED, class GEO>
+__device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* tmA, const CUtensorMap* tmB,
+                                               const GemmArgs& g, const FusedArgs* f, int ready_target, TileRange tr,
+                                               uint32_t& it, bool& ok) {
+    GemmCtrl* ctrl = c.ctrl;
+    constexpr uint32_t TX_BYTES = (FUSED && MODE == 1) ? G_B_BYTES : GEO::STAGE_BYTES + GEO::SCALE_BYTES;
+    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
+        const int wrow = __ldcg(g.tile_expert + m_tile) * g.w_rows_per_expert;
+        const float* a_sc = g.a_scale_t + static_cast<size_t>(m_tile) * TILE_M;
+        // claim the stage of pipeline iteration j: wait until its last reader has finished, announce the bytes
+        auto claim = [&](uint32_t j) -> bool {
+            const uint32_t s = j % GEO::STAGES, ph = (j / GEO::STAGES) & 1;
+            if (MODE == 1 && static_cast<int>(j) == g.fault_skip_it) return false;  // test hook: never filled
+            if (!mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, c.abort_flag, c.limit)) {
+                raise(ctrl, g.status, DEV_TIMEOUT_PRODUCER);
+                return false;
+            }
+            mbar_expect_tx(smem_u32(&ctrl->full[s]), TX_BYTES);
+            return true;
+        };
+        auto load_b = [&](uint32_t j, int kb) {
+            const uint32_t s = j % GEO::STAGES, bar = smem_u32(&ctrl->full[s]);
+            const uint32_t b_dst = c.smem_base + s * GEO::STAGE_BYTES + GEO::A_BYTES;
+            const int k0 = kb * G_BLOCK_K;
+            if (MODE == 1) {
+                const int gr = wrow + g.gate_row0 + n * 128, ur = wrow + g.up_row0 + n * 128;
+                tma_load_2d(b_dst, tmB, k0, gr, bar);
+                tma_load_2d(b_dst + G_B_BYTES / 4, tmB, k0, ur, bar);
+                tma_load_2d(b_dst + G_B_BYTES / 2, tmB, k0, gr + 64, bar);
+                tma_load_2d(b_dst + 3 * G_B_BYTES / 4, tmB, k0, ur + 64, bar);
+            } else {
+                const int br = wrow + n * G_TILE_N;
+                tma_load_2d(b_dst, tmB, k0, br, bar);
+                tma_load_2d(b_dst + G_B_BYTES / 2, tmB, k0, br + 128, bar);
+            }
+        };
+        auto load_a = [&](uint32_t j, int kb) {  // the A rows and their scales of the K-block
+            const uint32_t s = j % GEO::STAGES, bar = smem_u32(&ctrl->full[s]);
+            // (the scale slot is free: the ring exceeds the stages + accumulators the producer can be ahead
+            // of the epilogue)
+            bulk_load_1d(smem_u32(c.scale_ring + (j % GEO::SCALE_SLOTS) * GEO::A_ROWS),
+                         a_sc + static_cast<size_t>(kb) * g.row_cap, GEO::SCALE_BYTES, bar);
+            tma_load_2d(c.smem_base + s * GEO::STAGE_BYTES, tmA, kb * G_BLOCK_K, m_tile * TILE_M, bar);
+        };
+        int kb = 0;
+        if (FUSED && MODE == 2) {
+            // The tile's A rows are GEMM1's output and must have been stored; its weights need not wait for
+            // that, so the B tiles of the first K-blocks go out before the counter is looked at.
+            const int npre = g.num_kb < GEO::STAGES ? g.num_kb : GEO::STAGES;
+            for (int k = 0; k < npre && ok; ++k) {
+                ok = claim(it + k);
+                if (ok) load_b(it + k, k);
+            }
+            if (!ok) break;
+            if (!wait_counter(f->ready + m_tile, ready_target, c.abort_flag, c.limit)) {
+                raise(ctrl, g.status, DEV_TIMEOUT_READY);
+                ok = false;
+                break;
+            }
+            fence_proxy_async();  // the rows were stored by other CTAs' copy engines; order our copies behind the acquire
+            for (int k = 0; k < npre; ++k) load_a(it + k, k);
+            it += npre;
+            kb = npre;
+        }
+        for (; kb < g.num_kb && ok; ++kb, ++it) {
+            ok = claim(it);
+            if (!ok) break;
+            if (!(FUSED && MODE == 1)) load_a(it, kb);
+            load_b(it, kb);
+        }
+    }
+}
+
+// Before the producer thread may reach the end of the kernel every copy it issued has to have landed (bounded
+// wait).  On the regular path the MMA issuers have consumed all of them long ago and these waits fall through;
+// after an abort raised by any role they are what keeps the copy engine from writing into shared memory of a
+// CTA that has exited.
+template <class GEO>
+__device__ __forceinline__ void producer_drain(const Cta& c, int* status, uint32_t it) {
+    int zero = 0;
+    const uint32_t n_back = it < GEO::STAGES ? it : GEO::STAGES;
+    for (uint32_t j = it - n_back; j < it; ++j)
+        if (!mbar_wait(smem_u32(&c.ctrl->full[j % GEO::STAGES]), (j / GEO::STAGES) & 1, &zero, c.limit))
+            atomicCAS(status, DEV_OK, DEV_TIMEOUT_DRAIN);
+}
+
+// ---------------- MMA issuers (two threads) ----------------
+// Two threads share the issue work: `mine` = 0 takes the even K-blocks (TMEM buffer 0), 1 the odd ones (buffer
+// 1).  A commit only tracks the MMAs of its own thread, so while one thread pays for its commit and waits the
+// other keeps the tensor pipe fed.
+template <class GEO>
+__device__ __forceinline__ void issuer_tiles(const Cta& c, const GemmArgs& g, TileRange tr, uint32_t mine,
+                                             uint32_t& it, bool& ok) {
+    GemmCtrl* ctrl = c.ctrl;
+    const uint32_t idesc = umma_idesc_f8(TILE_M, G_TILE_N);
+    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+            if ((it & 1) != mine) continue;
+            const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
+            const uint32_t b = it & 1, bph = (it >> 1) & 1;
+            // The stage has normally landed long before the accumulator is handed back, so that
+            // wait comes first and only the hand-over itself is left on the critical path.
+            const uint32_t a_addr = c.smem_base + s * GEO::STAGE_BYTES;
+            const uint64_t a_desc = umma_desc_sw128(a_addr);  // 128 rows from here, fetched or not
+            const uint64_t b_desc = umma_desc_sw128(a_addr + GEO::A_BYTES);
+            const uint32_t d_tmem = c.tmem_base + b * G_TILE_N;
+            if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, c.abort_flag, c.limit)) {
+                raise(ctrl, g.status, DEV_TIMEOUT_MMA_SMEM);
+                ok = false;
+                break;
+            }
+            if (!mbar_wait(smem_u32(&ctrl->tmem_empty[b]), bph ^ 1, c.abort_flag, c.limit)) {
+                raise(ctrl, g.status, DEV_TIMEOUT_MMA_TMEM);
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+#pragma unroll
+            for (int k = 0; k < G_BLOCK_K / 32; ++k)  // 32 K-bytes per instruction: +2 in 16-B units
+                umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k > 0);
+            umma_commit(smem_u32(&ctrl->done[s]));
+        }
+    }
+}
+
+// After an abort: let issued MMAs retire before TMEM is released.
+__device__ __forceinline__ void issuer_drain(const Cta& c, uint32_t mine, bool ok) {
+    if (!ok || *c.abort_flag) {
+        umma_commit(smem_u32(&c.ctrl->drain_bar[mine]));
+        int zero = 0;
+        mbar_wait(smem_u32(&c.ctrl->drain_bar[mine]), 0, &zero, c.limit);
+    }
+}
+
+// ---------------- gather warp (fused kernel) ----------------
+// GEMM1 tiles: lane l copies 16-byte chunk (l & 7) of rows (l >> 3) + 4 i, i = 0..7, of every K-block from the
+// token-major input, and the scale of row l.  The stage uses the 128-byte swizzle of the TMA tiles: chunk c of
+// row r sits at r * 128 + ((c ^ (r & 7)) << 4), and r & 7 takes only two values per lane (i even / odd).  Rows
+// past the tile's valid rows are zero-filled; the stage holds only these 32 rows (see Geometry).  Each lane's arrival on full[s] is triggered by the completion of its copies.
+template <class GEO>
+__device__ __forceinline__ void gather_tiles(const Cta& c, const GemmArgs& g, const FusedArgs& f, TileRange tr,
+                                             uint32_t& it, bool& ok) {
+    GemmCtrl* ctrl = c.ctrl;
+    const int lane = c.lane, sub = lane >> 3, chunk = lane & 7;
+    const uint32_t dst_even = sub * 128 + ((chunk ^ sub) << 4);
+    const uint32_t dst_odd = sub * 128 + ((chunk ^ (sub + 4)) << 4);
+    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        const int m_tile = tile / g.n_tiles;
+        const int rows_valid = __ldcg(g.tile_rows + m_tile);
+        // token of row `lane` (scale copy) and source rows of this lane's eight chunks
+        const int my_tok = lane < rows_valid ? __ldcg(f.row_token + static_cast<size_t>(m_tile) * TILE_M + lane) : -1;
+        const uint8_t* src_row[GEO::A_ROWS / 4];
+#pragma unroll
+        for (int i = 0; i < GEO::A_ROWS / 4; ++i) {
+            const int t = __shfl_sync(0xffffffffu, my_tok, sub + 4 * i);
+            src_row[i] = t >= 0 ? f.hidden + static_cast<size_t>(t) * f.H + chunk * 16 : nullptr;
+        }
+        const float* sc_src = nullptr;
+        size_t sc_step = 0;
+        if (my_tok >= 0) {
+            sc_src = f.scale_layout ? f.hidden_scale + my_tok : f.hidden_scale + static_cast<size_t>(my_tok) * g.num_kb;
+            sc_step = f.scale_layout ? static_cast<size_t>(f.T) : 1;
+        }
+        for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+            const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, c.abort_flag, c.limit))) {
+                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_PRODUCER);
+                ok = false;
+                break;
+            }
+            const uint32_t a_dst = c.smem_base + s * GEO::STAGE_BYTES;
+#pragma unroll
+            for (int i = 0; i < GEO::A_ROWS / 4; ++i)
+                cp_async_16(a_dst + i * 512 + ((i & 1) ? dst_odd : dst_even),
+                            src_row[i] ? static_cast<const void*>(src_row[i] + kb * G_BLOCK_K)
+                                       : static_cast<const void*>(f.hidden),
+                            src_row[i] ? 16u : 0u);
+            cp_async_4(smem_u32(c.scale_ring + (it % GEO::SCALE_SLOTS) * GEO::A_ROWS + lane),
+                       sc_src ? static_cast<const void*>(sc_src + kb * sc_step) : static_cast<const void*>(f.hidden_scale),
+                       sc_src ? 4u : 0u);
+            cp_async_arrive_noinc(smem_u32(&ctrl->full[s]));
+        }
+    }
+}
+// GEMM2 tiles: the producer fetches everything; the lanes only keep the arrival count of full[s] uniform.
+template <class GEO>
+__device__ __forceinline__ void gather_idle_tiles(const Cta& c, const GemmArgs& g, TileRange tr, uint32_t& it, bool& ok) {
+    GemmCtrl* ctrl = c.ctrl;
+    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+            const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, c.abort_flag, c.limit))) {
+                ok = false;
+                break;
+            }
+            mbar_arrive(smem_u32(&ctrl->full[s]));
+        }
+    }
+}
+
+// Rendezvous of all epilogue threads (an mbarrier, because its wait is bounded: a plain barrier would hold the
+// arrived warps for ever if another warp had given up).  Orders the arrived threads' earlier writes before the
+// later reads of those that leave.  `n` counts the rendezvous of this thread so far.
+__device__ __forceinline__ bool epilogue_rendezvous(const Cta& c, uint32_t& n) {
+    const uint32_t bar = smem_u32(&c.ctrl->sync_bar[n & 1]);
+    mbar_arrive(bar);
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(bar, (n >> 1) & 1, c.abort_flag, c.limit));
+    ++n;
+    return ok;
+}
+
+// ---------------- epilogue warps ----------------
+// MODE 1: gate/up projection + SwiGLU + re-quantisation; tmOut describes the e4m3 output [row_cap, I] for
+//         64-byte x 32-row TMA stores.
+// MODE 2: down projection, bf16 rows out in the tile-blocked layout.
+// FUSED:  MODE 1 announces every stored tile in f->ready; MODE 2 counts the stored rows per (token, column
+//         tile) and combines the tokens it completes.
+template <int MODE, bool FUSED, class GEO>
+__device__ __forceinline__ void epilogue_tiles(const Cta& c, const CUtensorMap* tmOut, const GemmArgs& g,
+                                               const FusedArgs* f, TileRange tr, uint32_t& it, uint32_t& tile_iter,
+                                               uint32_t& sync_iter, bool& ok) {
+    GemmCtrl* ctrl = c.ctrl;
+    const int warp = c.warp, lane = c.lane;
+    const int widx = warp - 4;
+    const int half = widx >> 2;              // which 128-column half of the tile
+    const int quad = warp & 3;               // TMEM lane quadrant this warp may read
+    const int r_in_tile = quad * 32 + lane;  // accumulator row == TMEM lane
+    const uint32_t t_lane = c.tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * G_HALF_N;
+    const size_t row_cap = static_cast<size_t>(g.row_cap);
+    float* amax_x = c.amax_x;
+    // staging of this warp's GEMM1 rows; with the small geometry only the first row quadrant ever stores
+    uint8_t* stage = c.store_stage + (GEO::STORE_BYTES == G_EPI_WARPS * G_STORE_WARP_BYTES ? widx : half) * G_STORE_WARP_BYTES;
+    // row of the scale slot this thread reads (rows that are not fetched borrow the last fetched one: their
+    // accumulator rows are never stored)
+    const int scale_row = GEO::A_ROWS == TILE_M ? r_in_tile : (r_in_tile < GEO::A_ROWS ? r_in_tile : GEO::A_ROWS - 1);
+    const int num_kb = g.num_kb;
+    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
+        const int e = __ldcg(g.tile_expert + m_tile);
+        const int rows_valid = __ldcg(g.tile_rows + m_tile);
+        const size_t row = static_cast<size_t>(m_tile) * TILE_M + r_in_tile;
+        const int sblocks = g.w_rows_per_expert / 128;
+        // weight-scale rows of this thread's first / second 64 columns
+        const float* ws0;
+        const float* ws1;
+        if (MODE == 1) {
+            ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.gate_row0 / 128 + n) * num_kb;
+            ws1 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.up_row0 / 128 + n) * num_kb;
+        } else {
+            ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + 2 * n + half) * num_kb;
+            ws1 = ws0;
+        }
+        float acc[128];
+#pragma unroll
+        for (int j = 0; j < 128; ++j) acc[j] = 0.0f;
+
+        float s0 = __ldg(ws0), s1 = __ldg(ws1);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+            const float w0 = s0, w1 = s1;
+            if (kb + 1 < num_kb) {
+                s0 = __ldg(ws0 + kb + 1);
+                s1 = __ldg(ws1 + kb + 1);
+            }
+            const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1, buf = it & 1;
+            // Every lane polls (a single polling lane plus a broadcast was measured 2.5 % slower); the vote
+            // keeps the warp converged when a wait gives up: either all lanes go on or none does.
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph, c.abort_flag, c.limit))) {
+                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            // The MMA of this K-block has finished, hence its stage -- A, B and the scales -- had landed.
+            // (Fetching the scale earlier needs a barrier of its own per ring slot -- on full[s] this warp can
+            // be lapped by a whole phase -- and that extra barrier test per K-block was measured to cost the
+            // epilogue 110 clocks, 10 % of the kernel: barrier operations of a thread queue behind one another.)
+            const float sa = ld_shared_f32(c.scale_ring + (it % GEO::SCALE_SLOTS) * GEO::A_ROWS + scale_row);
+            const float f0 = sa * w0, f1 = sa * w1;
+            // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
+            const uint32_t col = t_lane + buf * G_TILE_N;
+            float v[64];
+            tmem_ld64(col, v);
+#pragma unroll
+            for (int j = 0; j < 64; ++j) acc[j] = fmaf(v[j], f0, acc[j]);
+            tmem_ld64(col + 64, v);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
+#pragma unroll
+            for (int j = 0; j < 64; ++j) acc[64 + j] = fmaf(v[j], f1, acc[64 + j]);
+        }
+        if (!ok) break;
+
+        if (MODE == 1) {
+            // The staging area of this warp was handed to the TMA engine at the end of the previous tile;
+            // by now (a whole tile later) that copy has long read it, so this wait does not stall.
+            if (lane == 0) bulk_wait_read_all();
+            __syncwarp();
+            const int sw = (lane >> 1) & 3;  // 64-byte swizzle: 16-byte chunk index ^= bits 7..8 of the address
+            // SwiGLU on this thread's 64 columns, then the row's 128-wide amax across the two halves
+            float cc[64];
+            float amax = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 64; ++j) {
+                // silu(g) * u with the hardware exp2 and reciprocal approximations (a few ulp): the
+                // tile's tail runs while the tensor pipe idles, so its instruction count matters.
+                const float gt = acc[j];
+                cc[j] = __fdividef(gt, 1.0f + __expf(-gt)) * acc[64 + j];
+                amax = fmaxf(amax, fabsf(cc[j]));
+            }
+            const uint32_t par = tile_iter & 1;
+            amax_x[(par * 2 + half) * TILE_M + r_in_tile] = amax;
+            const uint32_t xbar = smem_u32(&ctrl->amax_bar[par]);
+            mbar_arrive(xbar);
+            if (!__all_sync(0xffffffffu, mbar_wait(xbar, (tile_iter >> 1) & 1, c.abort_flag, c.limit))) {
+                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                ok = false;
+                break;
+            }
+            ++tile_iter;
+            amax = fmaxf(amax,
+                         *reinterpret_cast<volatile float*>(&amax_x[(par * 2 + (half ^ 1)) * TILE_M + r_in_tile]));
+            const float sc = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 448.0f);
+            const float inv_sc = __frcp_rn(sc);
+            if (quad * 32 < rows_valid) {
+                // e4m3 rows out: 32 rows x 64 bytes per warp, staged with the 64-byte swizzle, one TMA store
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int j = q * 16 + i * 4;
+                        const uint32_t lo = __nv_cvt_float2_to_fp8x2(
+                            make_float2(cc[j] * inv_sc, cc[j + 1] * inv_sc), __NV_SATFINITE, __NV_E4M3);
+                        const uint32_t hi = __nv_cvt_float2_to_fp8x2(
+                            make_float2(cc[j + 2] * inv_sc, cc[j + 3] * inv_sc), __NV_SATFINITE, __NV_E4M3);
+                        w[i] = lo | (hi << 16);
+                    }
+                    *reinterpret_cast<uint4*>(stage + lane * 64 + ((q ^ sw) << 4)) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_2d(tmOut, smem_u32(stage), n * 128 + half * 64, m_tile * TILE_M + quad * 32);
+                    bulk_commit_group();
+                }
+                if (half == 0 && r_in_tile < rows_valid)
+                    g.out_scale_t[static_cast<size_t>(n) * row_cap + row] = sc;
+            }
+            if (FUSED) {
+                // Announce the tile: the rows are in global memory once the bulk stores have completed (not
+                // merely been read); every thread's writes are fenced before the epilogue warps meet, and the
+                // announcing thread fences once more behind the barrier.
+                if (lane == 0) {
+                    bulk_wait_all();
+                    fence_proxy_async();
+                }
+                __threadfence();
+                if (!epilogue_rendezvous(c, sync_iter)) {
+                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                    ok = false;
+                    break;
+                }
+                if (warp == 4 && lane == 0) {
+                    __threadfence();
+                    atomicAdd(f->ready + m_tile, 1);
+                }
+            }
+        } else {
+            // bf16 rows out in a tile-blocked layout: block (row tile, column tile, half, quadrant) holds
+            // this warp's 32 rows x 128 columns as [8 column groups][32 rows][16 bf16], so every warp
+            // store instruction writes 1 KB of contiguous memory (32 bytes per lane).
+            if (quad * 32 < rows_valid) {
+                uint8_t* blk = reinterpret_cast<uint8_t*>(g.out_bf16) +
+                               (((static_cast<size_t>(m_tile) * g.n_tiles + n) * 2 + half) * 4 + quad) * 8192 +
+                               lane * 32;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    uint32_t w[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const __nv_bfloat162 pr = __floats2bfloat162_rn(acc[q * 16 + 2 * i], acc[q * 16 + 2 * i + 1]);
+                        w[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                    }
+                    st_global_v8(blk + q * 1024, w);
+                }
+            }
+            if (FUSED) {
+                // Stage 4 without a kernel of its own.  Once both halves of the tile are stored and fenced, the
+                // thread of each valid row bumps the counter of (its token, this column tile); whoever brings
+                // it to the token's number of local slots knows that all of the token's rows for these 256
+                // columns are in memory and sums them, in routing order, exactly as combine_kernel does.
+                __threadfence();
+                if (!epilogue_rendezvous(c, sync_iter)) {
+                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                    ok = false;
+                    break;
+                }
+                if (half == 0) {
+                    int tok = -1;
+                    bool last = false;
+                    if (r_in_tile < rows_valid) {
+                        tok = __ldcg(f->row_token + row);
+                        __threadfence();
+                        const int before = atomicAdd(f->tok_done + static_cast<size_t>(tok) * g.n_tiles + n, 1);
+                        last = before == __ldcg(f->tok_nlocal + tok) - 1;
+                    }
+                    uint32_t todo = __ballot_sync(0xffffffffu, last);
+                    if (todo) __threadfence();
+                    while (todo) {
+                        const int src = __ffs(todo) - 1;
+                        todo &= todo - 1;
+                        const int t = __shfl_sync(0xffffffffu, tok, src);
+                        // lane l owns columns n*256 + 8 l .. + 8: half of the 32-byte group n*16 + l/2
+                        float o[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) o[i] = 0.0f;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const int r = __ldcg(f->slot_to_row + t * 8 + j);
+                            if (r < 0) continue;
+                            const float wj = __ldcg(f->topk_w + t * 8 + j);
+                            const uint4 u = __ldcg(reinterpret_cast<const uint4*>(
+                                reinterpret_cast<const uint8_t*>(g.out_bf16) + y_block_offset(r, n * 16 + (lane >> 1), g.n_tiles) +
+                                (lane & 1) * 16));
+                            const uint32_t uu[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                o[2 * i] = fmaf(wj, __uint_as_float(uu[i] << 16), o[2 * i]);
+                                o[2 * i + 1] = fmaf(wj, __uint_as_float(uu[i] & 0xffff0000u), o[2 * i + 1]);
+                            }
+                        }
+                        uint32_t p[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const __nv_bfloat162 pr = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+                            p[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                        }
+                        *reinterpret_cast<uint4*>(f->out + static_cast<size_t>(t) * f->H + n * G_TILE_N + lane * 8) =
+                            make_uint4(p[0], p[1], p[2], p[3]);
+                    }
+                }
+            }
+        }
+    }
+}
+
+// One GEMM per launch.
+template <int MODE>
+__global__ void __launch_bounds__(G_THREADS, 1)
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmOut, const GemmArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    using GEO = GeomFull;
+    Cta c;
+    gemm_cta_setup<GEO>(c, smem_raw, 1);
+    if (c.warp == 0 && c.lane == 0) {
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
         if (MODE == 1) tma_prefetch_desc(&tmOut);
@@ -139,273 +671,106 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // scales below were written by the kernels before this one.
     pdl_launch_dependents();
     pdl_wait();
-    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&ctrl->tmem_slot);
+    c.tmem_base = *reinterpret_cast<volatile uint32_t*>(&c.ctrl->tmem_slot);
+    c.limit = g.wait_limit;
     // (the tables come from the kernels before this one, which may still be resident: coherent loads)
-    const int num_tiles = __ldcg(g.num_m_tiles) * g.n_tiles;
-    const int num_kb = g.num_kb;
-    const long long limit = g.wait_limit;
+    const TileRange tr = {static_cast<int>(blockIdx.x), __ldcg(g.num_m_tiles) * g.n_tiles, static_cast<int>(gridDim.x)};
+    uint32_t it = 0;
+    bool ok = true;
 
-    if (warp < 4) {
+    if (c.warp < 4) {
         reg_dealloc<40>();
-        if (warp == 0 && lane == 0) {
-            // ---------------- TMA producer ----------------
-            uint32_t it = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
-                const int wrow = __ldcg(g.tile_expert + m_tile) * g.w_rows_per_expert;
-                const float* a_sc = g.a_scale_t + static_cast<size_t>(m_tile) * TILE_M;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1;
-                    if (static_cast<int>(it) == g.fault_skip_it) {  // test hook: this stage is never filled
-                        ok = false;
-                        break;
-                    }
-                    if (!mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, abort_flag, limit)) {
-                        raise(ctrl, g.status, DEV_TIMEOUT_PRODUCER);
-                        ok = false;
-                        break;
-                    }
-                    const uint32_t bar = smem_u32(&ctrl->full[s]);
-                    const uint32_t a_dst = smem_base + s * G_STAGE_BYTES, b_dst = a_dst + G_A_BYTES;
-                    const int k0 = kb * G_BLOCK_K;
-                    // (the scale slot is free: 8 slots exceed the 4 stages + 2 accumulators the producer can be
-                    // ahead of the epilogue)
-                    mbar_expect_tx(bar, G_STAGE_BYTES + G_SCALE_BYTES);
-                    bulk_load_1d(smem_u32(scale_ring + (it % G_SCALE_RING) * TILE_M),
-                                 a_sc + static_cast<size_t>(kb) * g.row_cap, G_SCALE_BYTES, bar);
-                    tma_load_2d(a_dst, &tmA, k0, m_tile * TILE_M, bar);
-                    if (MODE == 1) {
-                        const int gr = wrow + g.gate_row0 + n * 128, ur = wrow + g.up_row0 + n * 128;
-                        tma_load_2d(b_dst, &tmB, k0, gr, bar);
-                        tma_load_2d(b_dst + G_B_BYTES / 4, &tmB, k0, ur, bar);
-                        tma_load_2d(b_dst + G_B_BYTES / 2, &tmB, k0, gr + 64, bar);
-                        tma_load_2d(b_dst + 3 * G_B_BYTES / 4, &tmB, k0, ur + 64, bar);
-                    } else {
-                        const int br = wrow + n * G_TILE_N;
-                        tma_load_2d(b_dst, &tmB, k0, br, bar);
-                        tma_load_2d(b_dst + G_B_BYTES / 2, &tmB, k0, br + 128, bar);
-                    }
-                }
-            }
-            {
-                // Before this thread may reach the end of the kernel every copy it issued has to have landed
-                // (bounded wait).  On the regular path the MMA issuers have consumed all of them long ago and
-                // these waits fall through; after an abort raised by any role they are what keeps the
-                // copy engine from writing into shared memory of a CTA that has exited.
-                int zero = 0;
-                const uint32_t n_back = it < G_STAGES ? it : G_STAGES;
-                for (uint32_t j = it - n_back; j < it; ++j)
-                    if (!mbar_wait(smem_u32(&ctrl->full[j % G_STAGES]), (j / G_STAGES) & 1, &zero, limit))
-                        atomicCAS(g.status, DEV_OK, DEV_TIMEOUT_DRAIN);
-            }
-        } else if ((warp == 1 || warp == 2) && lane == 0) {
-            // ---------------- MMA issuers ----------------
-            // Two threads share the issue work: warp 1 takes the even K-blocks (TMEM buffer 0), warp 2 the
-            // odd ones (buffer 1).  A commit only tracks the MMAs of its own thread, so while one thread
-            // pays for its commit and waits the other keeps the tensor pipe fed.
-            const uint32_t idesc = umma_idesc_f8(TILE_M, G_TILE_N);
-            const uint32_t mine = warp - 1;
-            uint32_t it = 0;
-            bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                    if ((it & 1) != mine) continue;
-                    const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1;
-                    const uint32_t b = it & 1, bph = (it >> 1) & 1;
-                    // The stage has normally landed long before the accumulator is handed back, so that
-                    // wait comes first and only the hand-over itself is left on the critical path.
-                    const uint32_t a_addr = smem_base + s * G_STAGE_BYTES;
-                    const uint64_t a_desc = umma_desc_sw128(a_addr);
-                    const uint64_t b_desc = umma_desc_sw128(a_addr + G_A_BYTES);
-                    const uint32_t d_tmem = tmem_base + b * G_TILE_N;
-                    if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, abort_flag, limit)) {
-                        raise(ctrl, g.status, DEV_TIMEOUT_MMA_SMEM);
-                        ok = false;
-                        break;
-                    }
-                    if (!mbar_wait(smem_u32(&ctrl->tmem_empty[b]), bph ^ 1, abort_flag, limit)) {
-                        raise(ctrl, g.status, DEV_TIMEOUT_MMA_TMEM);
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < G_BLOCK_K / 32; ++k)  // 32 K-bytes per instruction: +2 in 16-B units
-                        umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k > 0);
-                    umma_commit(smem_u32(&ctrl->done[s]));
-                }
-            }
-            if (!ok || *abort_flag) {  // let issued MMAs retire before TMEM is released
-                umma_commit(smem_u32(&ctrl->drain_bar[mine]));
-                int zero = 0;
-                mbar_wait(smem_u32(&ctrl->drain_bar[mine]), 0, &zero, limit);
-            }
+        if (c.warp == 0 && c.lane == 0) {
+            producer_tiles<MODE, false, GEO>(c, &tmA, &tmB, g, nullptr, 0, tr, it, ok);
+            producer_drain<GEO>(c, g.status, it);
+        } else if ((c.warp == 1 || c.warp == 2) && c.lane == 0) {
+            issuer_tiles<GEO>(c, g, tr, c.warp - 1, it, ok);
+            issuer_drain(c, c.warp - 1, ok);
         }
     } else {
-        // ---------------- epilogue warps ----------------
         reg_alloc<232>();
-        const int widx = warp - 4;
-        const int half = widx >> 2;              // which 128-column half of the tile
-        const int quad = warp & 3;               // TMEM lane quadrant this warp may read
-        const int r_in_tile = quad * 32 + lane;  // accumulator row == TMEM lane
-        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * G_HALF_N;
-        const size_t row_cap = static_cast<size_t>(g.row_cap);
-        float* amax_x = reinterpret_cast<float*>(store_stage + G_STORE_BYTES);  // [2][2][TILE_M], GEMM1 only
-        uint8_t* stage = store_stage + widx * G_STORE_WARP_BYTES;
-        uint32_t it = 0, tile_iter = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tile_iter) {
-            const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
-            const int e = __ldcg(g.tile_expert + m_tile);
-            const int rows_valid = __ldcg(g.tile_rows + m_tile);
-            const size_t row = static_cast<size_t>(m_tile) * TILE_M + r_in_tile;
-            const int sblocks = g.w_rows_per_expert / 128;
-            // weight-scale rows of this thread's first / second 64 columns
-            const float* ws0;
-            const float* ws1;
-            if (MODE == 1) {
-                ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.gate_row0 / 128 + n) * num_kb;
-                ws1 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.up_row0 / 128 + n) * num_kb;
-            } else {
-                ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + 2 * n + half) * num_kb;
-                ws1 = ws0;
-            }
-            float acc[128];
-#pragma unroll
-            for (int j = 0; j < 128; ++j) acc[j] = 0.0f;
-
-            float s0 = __ldg(ws0), s1 = __ldg(ws1);
-            for (int kb = 0; kb < num_kb; ++kb, ++it) {
-                const float w0 = s0, w1 = s1;
-                if (kb + 1 < num_kb) {
-                    s0 = __ldg(ws0 + kb + 1);
-                    s1 = __ldg(ws1 + kb + 1);
-                }
-                const uint32_t s = it % G_STAGES, ph = (it / G_STAGES) & 1, buf = it & 1;
-                // Every lane polls (a single polling lane plus a broadcast was measured 2.5 % slower); the vote
-                // keeps the warp converged when a wait gives up: either all lanes go on or none does.
-                if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph, abort_flag, limit))) {
-                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                    ok = false;
-                    break;
-                }
-                tc_fence_after();
-                // The MMA of this K-block has finished, hence its stage -- A, B and the scales -- had landed.
-                // (Fetching the scale earlier needs a barrier of its own per ring slot -- on full[s] this warp can
-                // be lapped by a whole phase -- and that extra barrier test per K-block was measured to cost the
-                // epilogue 110 clocks, 10 % of the kernel: barrier operations of a thread queue behind one another.)
-                const float sa = ld_shared_f32(scale_ring + (it % G_SCALE_RING) * TILE_M + r_in_tile);
-                const float f0 = sa * w0, f1 = sa * w1;
-                // GEMM1: of this warpgroup's 128 columns, [0,64) are gate and [64,128) the matching up columns.
-                const uint32_t col = t_lane + buf * G_TILE_N;
-                float v[64];
-                tmem_ld64(col, v);
-#pragma unroll
-                for (int j = 0; j < 64; ++j) acc[j] = fmaf(v[j], f0, acc[j]);
-                tmem_ld64(col + 64, v);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
-#pragma unroll
-                for (int j = 0; j < 64; ++j) acc[64 + j] = fmaf(v[j], f1, acc[64 + j]);
-            }
-            if (!ok) break;
-
-            // The staging area of this warp was handed to the TMA engine at the end of the previous tile;
-            // by now (a whole tile later) that copy has long read it, so this wait does not stall.
-            if (lane == 0) bulk_wait_read_all();
-            __syncwarp();
-            const int sw = (lane >> 1) & 3;  // 64-byte swizzle: 16-byte chunk index ^= bits 7..8 of the address
-
-            if (MODE == 1) {
-                // SwiGLU on this thread's 64 columns, then the row's 128-wide amax across the two halves
-                float c[64];
-                float amax = 0.0f;
-#pragma unroll
-                for (int j = 0; j < 64; ++j) {
-                    // silu(g) * u with the hardware exp2 and reciprocal approximations (a few ulp): the
-                    // tile's tail runs while the tensor pipe idles, so its instruction count matters.
-                    const float gt = acc[j];
-                    c[j] = __fdividef(gt, 1.0f + __expf(-gt)) * acc[64 + j];
-                    amax = fmaxf(amax, fabsf(c[j]));
-                }
-                const uint32_t par = tile_iter & 1;
-                amax_x[(par * 2 + half) * TILE_M + r_in_tile] = amax;
-                const uint32_t xbar = smem_u32(&ctrl->amax_bar[par]);
-                mbar_arrive(xbar);
-                if (!__all_sync(0xffffffffu, mbar_wait(xbar, (tile_iter >> 1) & 1, abort_flag, limit))) {
-                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                    break;
-                }
-                amax = fmaxf(amax,
-                             *reinterpret_cast<volatile float*>(&amax_x[(par * 2 + (half ^ 1)) * TILE_M + r_in_tile]));
-                const float sc = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 448.0f);
-                const float inv_sc = __frcp_rn(sc);
-                if (quad * 32 < rows_valid) {
-                    // e4m3 rows out: 32 rows x 64 bytes per warp, staged with the 64-byte swizzle, one TMA store
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const int j = q * 16 + i * 4;
-                            const uint32_t lo = __nv_cvt_float2_to_fp8x2(
-                                make_float2(c[j] * inv_sc, c[j + 1] * inv_sc), __NV_SATFINITE, __NV_E4M3);
-                            const uint32_t hi = __nv_cvt_float2_to_fp8x2(
-                                make_float2(c[j + 2] * inv_sc, c[j + 3] * inv_sc), __NV_SATFINITE, __NV_E4M3);
-                            w[i] = lo | (hi << 16);
-                        }
-                        *reinterpret_cast<uint4*>(stage + lane * 64 + ((q ^ sw) << 4)) =
-                            make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&tmOut, smem_u32(stage), n * 128 + half * 64, m_tile * TILE_M + quad * 32);
-                        bulk_commit_group();
-                    }
-                    if (half == 0 && r_in_tile < rows_valid)
-                        g.out_scale_t[static_cast<size_t>(n) * row_cap + row] = sc;
-                }
-            } else {
-                // bf16 rows out in a tile-blocked layout: block (row tile, column tile, half, quadrant) holds
-                // this warp's 32 rows x 128 columns as [8 column groups][32 rows][16 bf16], so every warp
-                // store instruction writes 1 KB of contiguous memory (32 bytes per lane).
-                if (quad * 32 < rows_valid) {
-                    uint8_t* blk = reinterpret_cast<uint8_t*>(g.out_bf16) +
-                                   (((static_cast<size_t>(m_tile) * g.n_tiles + n) * 2 + half) * 4 + quad) * 8192 +
-                                   lane * 32;
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        uint32_t w[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const __nv_bfloat162 pr = __floats2bfloat162_rn(acc[q * 16 + 2 * i], acc[q * 16 + 2 * i + 1]);
-                            w[i] = *reinterpret_cast<const uint32_t*>(&pr);
-                        }
-                        st_global_v8(blk + q * 1024, w);
-                    }
-                }
-            }
-        }
-        if (lane == 0) bulk_wait_all();
+        uint32_t tile_iter = 0, sync_iter = 0;
+        epilogue_tiles<MODE, false, GEO>(c, &tmOut, g, nullptr, tr, it, tile_iter, sync_iter, ok);
+        if (c.lane == 0) bulk_wait_all();
     }
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (c.warp == 1) {
         __syncwarp();
-        tmem_dealloc(tmem_base, G_TMEM_COLS);
+        tmem_dealloc(c.tmem_base, G_TMEM_COLS);
     }
 }
 
-// Byte offset of the 32-byte group holding columns [16*c16, 16*c16+16) of padded row r in the
-// tile-blocked bf16 output of GEMM2 (n_tiles = H / 256 column tiles).
-__host__ __device__ __forceinline__ size_t y_block_offset(int r, int c16, int n_tiles) {
-    const int m_tile = r / TILE_M, quad = (r % TILE_M) / 32, lane = r % 32;
-    const int n = c16 / 16, half = (c16 % 16) / 8, q = c16 % 8;
-    return (((static_cast<size_t>(m_tile) * n_tiles + n) * 2 + half) * 4 + quad) * 8192 + q * 1024 + lane * 32;
+// Gather + GEMM1 + GEMM2 + combine in one launch for batches of at most F_MAX_TOKENS tokens (see the head of
+// this file).  tmA2 / tmOut describe GEMM1's output buffer for loads (32-row boxes) / stores, tmB1 / tmB2 the
+// two weight tensors.
+__global__ void __launch_bounds__(G_THREADS, 1)
+fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB1,
+                   const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmOut,
+                   const GemmArgs g1, const GemmArgs g2, const FusedArgs f) {
+    extern __shared__ uint8_t smem_raw[];
+    using GEO = GeomSmall;
+    Cta c;
+    gemm_cta_setup<GEO>(c, smem_raw, 33);  // the producer's arrival plus the 32 lanes of the gather warp
+    if (c.warp == 0 && c.lane == 0) {
+        tma_prefetch_desc(&tmA2);
+        tma_prefetch_desc(&tmB1);
+        tma_prefetch_desc(&tmB2);
+        tma_prefetch_desc(&tmOut);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    pdl_launch_dependents();
+    pdl_wait();
+    c.tmem_base = *reinterpret_cast<volatile uint32_t*>(&c.ctrl->tmem_slot);
+    c.limit = g1.wait_limit;
+
+    // tokens without a local expert: their output rows are zeros, written here by the CTAs in turn
+    for (int t = blockIdx.x; t < f.T; t += gridDim.x)
+        if (__ldcg(f.tok_nlocal + t) == 0)
+            for (int i = threadIdx.x; i < f.H / 8; i += blockDim.x)
+                reinterpret_cast<uint4*>(f.out + static_cast<size_t>(t) * f.H)[i] = make_uint4(0u, 0u, 0u, 0u);
+
+    // The CTA's work list: its GEMM1 tiles, then its GEMM2 tiles; the grid-strided numbering runs on from one
+    // phase into the next, so the CTAs that had no GEMM1 tile take the first GEMM2 tiles.
+    const int grid = static_cast<int>(gridDim.x), m_tiles = __ldcg(g1.num_m_tiles);
+    const int n1 = m_tiles * g1.n_tiles, n2 = m_tiles * g2.n_tiles;
+    const TileRange tr1 = {static_cast<int>(blockIdx.x), n1, grid};
+    const TileRange tr2 = {((static_cast<int>(blockIdx.x) - n1) % grid + grid) % grid, n2, grid};
+    uint32_t it = 0;
+    bool ok = true;
+
+    if (c.warp < 4) {
+        reg_dealloc<40>();
+        if (c.warp == 0 && c.lane == 0) {
+            producer_tiles<1, true, GEO>(c, &tmA2, &tmB1, g1, &f, 0, tr1, it, ok);
+            producer_tiles<2, true, GEO>(c, &tmA2, &tmB2, g2, &f, g1.n_tiles, tr2, it, ok);
+            producer_drain<GEO>(c, g1.status, it);
+        } else if ((c.warp == 1 || c.warp == 2) && c.lane == 0) {
+            issuer_tiles<GEO>(c, g1, tr1, c.warp - 1, it, ok);
+            issuer_tiles<GEO>(c, g2, tr2, c.warp - 1, it, ok);
+            issuer_drain(c, c.warp - 1, ok);
+        } else if (c.warp == 3) {
+            gather_tiles<GEO>(c, g1, f, tr1, it, ok);
+            gather_idle_tiles<GEO>(c, g2, tr2, it, ok);
+            cp_async_wait_all();  // nothing may still be landing in shared memory when the CTA exits
+        }
+    } else {
+        reg_alloc<232>();
+        uint32_t tile_iter = 0, sync_iter = 0;
+        epilogue_tiles<1, true, GEO>(c, &tmOut, g1, &f, tr1, it, tile_iter, sync_iter, ok);
+        epilogue_tiles<2, true, GEO>(c, &tmOut, g2, &f, tr2, it, tile_iter, sync_iter, ok);
+        if (c.lane == 0) bulk_wait_all();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (c.warp == 1) {
+        __syncwarp();
+        tmem_dealloc(c.tmem_base, G_TMEM_COLS);
+    }
 }
 
 }  // namespace moe

@@ -30,7 +30,7 @@ inline size_t align_up(size_t x, size_t a = WS_ALIGN) { return (x + a - 1) / a *
 
 struct WsLayout {
     size_t topk_idx, topk_w, block_hist, expert_count, expert_offset, padded_offset, tile_expert, tile_rows,
-        num_m_tiles, slot_to_row, row_to_slot, row_token, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
+        num_m_tiles, slot_to_row, row_to_slot, row_token, tok_nlocal, ready, tok_done, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
         stage_scale, stage_logits, stage_out, total;
     int row_cap, max_m_tiles, max_blocks;
 };
@@ -62,6 +62,9 @@ WsLayout make_layout(const moe_fp8_config& c) {
     L.slot_to_row = take(slots * 4);
     L.row_to_slot = take(slots * 4);
     L.row_token = take(rc * 4);
+    L.tok_nlocal = take(Tm * 4);
+    L.ready = take(std::max<size_t>(EL, 1) * 4);
+    L.tok_done = take(static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N) * 4);
     L.status = take(8);  // device status word, then the ticket counter of route_permute_kernel
     L.a1 = take(rc * H);
     L.a1_scale_t = take(rc * (H / 128) * 4);
@@ -78,6 +81,8 @@ WsLayout make_layout(const moe_fp8_config& c) {
 
 }  // namespace
 
+constexpr int NUM_STAGES_MAX = 9;
+
 struct moe_fp8_handle_s {
     moe_fp8_config cfg;
     WsLayout L;
@@ -88,14 +93,15 @@ struct moe_fp8_handle_s {
     uint8_t* ws;
     size_t ws_bytes;
     EncodeTiledFn encode;
-    CUtensorMap tm_a1, tm_a2, tm_a2_store, tm_w13, tm_w2;
+    CUtensorMap tm_a1, tm_a2, tm_a2_small, tm_a2_store, tm_w13, tm_w2;
     const void* w13_cached;
     const void* w2_cached;
     bool stage_timing;
     bool stage_times_valid;
     int fault_skip_it;         // test hook, see moe_fp8_debug_set_fault
     long long fault_wait_limit;
-    cudaEvent_t ev[9];
+    cudaEvent_t ev[NUM_STAGES_MAX + 1];
+    bool small_fusion;         // batches of at most F_MAX_TOKENS tokens take the single fused kernel
 };
 
 namespace {
@@ -154,13 +160,17 @@ PermuteMeta meta_of(moe_fp8_handle_t h) {
     m.slot_to_row = at<int>(h, h->L.slot_to_row);
     m.row_to_slot = at<int>(h, h->L.row_to_slot);
     m.row_token = at<int>(h, h->L.row_token);
+    m.tok_nlocal = at<int>(h, h->L.tok_nlocal);
+    m.ready = at<int>(h, h->L.ready);
+    m.tok_done = at<int>(h, h->L.tok_done);
+    m.done_cols = 0;
     return m;
 }
 
 constexpr int PDL_MAX_TOKENS = 2048;
-constexpr int NUM_STAGES = 8;
+constexpr int NUM_STAGES = 9;
 const char* const STAGE_NAMES[NUM_STAGES] = {"route_topk", "count", "scan", "place", "gather_rows",
-                                             "gemm1_swiglu_quant", "gemm2", "combine"};
+                                             "gemm1_swiglu_quant", "gemm2", "combine", "fused_small"};
 
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -234,9 +244,11 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
     if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) return MOE_FP8_ERR_CUDA;
 
-    e = cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    e = cudaFuncSetAttribute(grouped_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, GeomFull::SMEM_BYTES);
     if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
-    e = cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM_BYTES);
+    e = cudaFuncSetAttribute(grouped_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, GeomFull::SMEM_BYTES);
+    if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
+    e = cudaFuncSetAttribute(fused_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GeomSmall::SMEM_BYTES);
     if (e != cudaSuccess) return MOE_FP8_ERR_CUDA;
     e = cudaFuncSetAttribute(router_logits_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(router_smem_bytes(4, 4)));
@@ -251,6 +263,7 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     h->cfg = *cfg;
     h->L = make_layout(*cfg);
     h->sm_count = sms;
+    h->small_fusion = true;
     h->fault_skip_it = -1;
     h->fault_wait_limit = WAIT_LIMIT_CLOCKS;
     h->encode = reinterpret_cast<EncodeTiledFn>(fn);
@@ -281,6 +294,8 @@ int moe_fp8_set_workspace(moe_fp8_handle_t h, void* ws, size_t bytes) {
     if (!encode_2d(h, &h->tm_a1, h->ws + h->L.a1, h->L.row_cap, h->cfg.hidden, 1, 128, TILE_M,
                    CU_TENSOR_MAP_SWIZZLE_128B) ||
         !encode_2d(h, &h->tm_a2, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate, 1, 128, TILE_M,
+                   CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !encode_2d(h, &h->tm_a2_small, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate, 1, 128, GeomSmall::A_ROWS,
                    CU_TENSOR_MAP_SWIZZLE_128B) ||
         !encode_2d(h, &h->tm_a2_store, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate, 1, 64, 32,
                    CU_TENSOR_MAP_SWIZZLE_64B)) {
@@ -357,6 +372,8 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     } while (0)
     h->stage_times_valid = false;
     mark();
+    const bool fused = h->small_fusion && T <= F_MAX_TOKENS;
+    if (fused) m.done_cols = H / G_TILE_N;
 
     if (T <= P_TAIL_MAX_TOKENS) {  // routing in parallel blocks, the last one to finish does stage 2
         const int grid = min((T + 7) / 8, h->sm_count * 8);
@@ -384,64 +401,89 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
                    static_cast<const int*>(topk_idx), m, status);
         mark();
     }
-    {  // stage 2, continued: gather
-        const long long row_bound = static_cast<long long>(T) * 8 + static_cast<long long>(EL) * (TILE_M - 1);
-        const int grid = static_cast<int>(std::min<long long>((row_bound + 7) / 8, h->sm_count * 8LL));
-        MOE_LAUNCH(gather_rows_kernel, grid, 256, 0, stream, pdl, H, row_cap, c.hidden_scale_layout, T,
-                   static_cast<const uint8_t*>(hidden_fp8), hidden_scale, m, a1, a1_scale_t);
+    // the two GEMMs' arguments
+    GemmArgs g1, g2;
+    memset(&g1, 0, sizeof(g1));
+    g1.num_kb = H / 128;
+    g1.n_tiles = I / 128;
+    g1.w_rows_per_expert = 2 * I;
+    g1.row_cap = row_cap;
+    g1.out_cols = I;
+    g1.gate_row0 = c.gate_first ? 0 : I;
+    g1.up_row0 = c.gate_first ? I : 0;
+    g1.num_m_tiles = m.num_m_tiles;
+    g1.tile_expert = m.tile_expert;
+    g1.tile_rows = m.tile_rows;
+    g1.a_scale_t = a1_scale_t;
+    g1.w_scale = w13_scale;
+    g1.out_fp8 = a2;
+    g1.out_scale_t = a2_scale_t;
+    g1.status = status;
+    g1.wait_limit = h->fault_wait_limit;
+    g1.fault_skip_it = h->fault_skip_it;
+    memset(&g2, 0, sizeof(g2));
+    g2.num_kb = I / 128;
+    g2.n_tiles = H / G_TILE_N;
+    g2.w_rows_per_expert = H;
+    g2.row_cap = row_cap;
+    g2.out_cols = H;
+    g2.num_m_tiles = m.num_m_tiles;
+    g2.tile_expert = m.tile_expert;
+    g2.tile_rows = m.tile_rows;
+    g2.a_scale_t = a2_scale_t;
+    g2.w_scale = w2_scale;
+    g2.out_bf16 = y;
+    g2.status = status;
+    g2.wait_limit = h->fault_wait_limit;
+    g2.fault_skip_it = -1;
+
+    if (fused) {
+        // stages 2 (gather), 3 and 4 in one launch
+        FusedArgs f;
+        memset(&f, 0, sizeof(f));
+        f.T = T;
+        f.H = H;
+        f.scale_layout = c.hidden_scale_layout;
+        f.hidden = static_cast<const uint8_t*>(hidden_fp8);
+        f.hidden_scale = hidden_scale;
+        f.row_token = m.row_token;
+        f.slot_to_row = m.slot_to_row;
+        f.topk_w = topk_w;
+        f.tok_nlocal = m.tok_nlocal;
+        f.ready = m.ready;
+        f.tok_done = m.tok_done;
+        f.out = static_cast<__nv_bfloat16*>(out);
+        mark();  // gather_rows
+        mark();  // gemm1
+        mark();  // gemm2
+        mark();  // combine
+        MOE_LAUNCH(fused_small_kernel, h->sm_count, G_THREADS, GeomSmall::SMEM_BYTES, stream, pdl, h->tm_a2_small,
+                   h->tm_w13, h->tm_w2, h->tm_a2_store, g1, g2, f);
         mark();
-    }
-    {  // stage 3a: GEMM1 + SwiGLU + re-quantisation
-        GemmArgs g;
-        memset(&g, 0, sizeof(g));
-        g.num_kb = H / 128;
-        g.n_tiles = I / 128;
-        g.w_rows_per_expert = 2 * I;
-        g.row_cap = row_cap;
-        g.out_cols = I;
-        g.gate_row0 = c.gate_first ? 0 : I;
-        g.up_row0 = c.gate_first ? I : 0;
-        g.num_m_tiles = m.num_m_tiles;
-        g.tile_expert = m.tile_expert;
-        g.tile_rows = m.tile_rows;
-        g.a_scale_t = a1_scale_t;
-        g.w_scale = w13_scale;
-        g.out_fp8 = a2;
-        g.out_scale_t = a2_scale_t;
-        g.status = status;
-        g.wait_limit = h->fault_wait_limit;
-        g.fault_skip_it = h->fault_skip_it;
-        MOE_LAUNCH(grouped_gemm_kernel<1>, h->sm_count, G_THREADS, G_SMEM_BYTES, stream, pdl, h->tm_a1, h->tm_w13,
-                   h->tm_a2_store, g);
+    } else {
+        {  // stage 2, continued: gather
+            const long long row_bound = static_cast<long long>(T) * 8 + static_cast<long long>(EL) * (TILE_M - 1);
+            const int grid = static_cast<int>(std::min<long long>((row_bound + 7) / 8, h->sm_count * 8LL));
+            MOE_LAUNCH(gather_rows_kernel, grid, 256, 0, stream, pdl, H, row_cap, c.hidden_scale_layout, T,
+                       static_cast<const uint8_t*>(hidden_fp8), hidden_scale, m, a1, a1_scale_t);
+            mark();
+        }
+        // stage 3a: GEMM1 + SwiGLU + re-quantisation
+        MOE_LAUNCH(grouped_gemm_kernel<1>, h->sm_count, G_THREADS, GeomFull::SMEM_BYTES, stream, pdl, h->tm_a1,
+                   h->tm_w13, h->tm_a2_store, g1);
         mark();
-    }
-    {  // stage 3b: GEMM2
-        GemmArgs g;
-        memset(&g, 0, sizeof(g));
-        g.num_kb = I / 128;
-        g.n_tiles = H / G_TILE_N;
-        g.w_rows_per_expert = H;
-        g.row_cap = row_cap;
-        g.out_cols = H;
-        g.num_m_tiles = m.num_m_tiles;
-        g.tile_expert = m.tile_expert;
-        g.tile_rows = m.tile_rows;
-        g.a_scale_t = a2_scale_t;
-        g.w_scale = w2_scale;
-        g.out_bf16 = y;
-        g.status = status;
-        g.wait_limit = h->fault_wait_limit;
-        g.fault_skip_it = -1;
-        MOE_LAUNCH(grouped_gemm_kernel<2>, h->sm_count, G_THREADS, G_SMEM_BYTES, stream, pdl, h->tm_a2, h->tm_w2,
-                   h->tm_a2_store, g);
+        // stage 3b: GEMM2
+        MOE_LAUNCH(grouped_gemm_kernel<2>, h->sm_count, G_THREADS, GeomFull::SMEM_BYTES, stream, pdl, h->tm_a2,
+                   h->tm_w2, h->tm_a2_store, g2);
         mark();
-    }
-    {  // stage 4: weighted combine back to token order
-        const int grid = min(T, h->sm_count * 16);
-        MOE_LAUNCH(combine_kernel, grid, 256, 0, stream, pdl, T, H, static_cast<const int*>(m.slot_to_row),
-                   static_cast<const float*>(topk_w), reinterpret_cast<const uint8_t*>(y),
-                   static_cast<__nv_bfloat16*>(out));
-        mark();
+        {  // stage 4: weighted combine back to token order
+            const int grid = min(T, h->sm_count * 16);
+            MOE_LAUNCH(combine_kernel, grid, 256, 0, stream, pdl, T, H, static_cast<const int*>(m.slot_to_row),
+                       static_cast<const float*>(topk_w), reinterpret_cast<const uint8_t*>(y),
+                       static_cast<__nv_bfloat16*>(out));
+            mark();
+        }
+        mark();  // fused_small (not used on this path)
     }
 #undef MOE_LAUNCH
     const cudaError_t e = cudaGetLastError();
@@ -455,6 +497,12 @@ int moe_fp8_debug_set_fault(moe_fp8_handle_t h, int skip_iteration, long long wa
     if (!h || wait_clocks < 0) return MOE_FP8_ERR_BAD_ARG;
     h->fault_skip_it = skip_iteration < 0 ? -1 : skip_iteration;
     h->fault_wait_limit = wait_clocks == 0 ? WAIT_LIMIT_CLOCKS : wait_clocks;
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_set_small_batch_fusion(moe_fp8_handle_t h, int enable) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    h->small_fusion = enable != 0;
     return MOE_FP8_OK;
 }
 

@@ -30,6 +30,11 @@ struct PermuteMeta {
     int* slot_to_row;    // [T*8] padded row of each slot, -1 when the slot's expert is not local
     int* row_to_slot;    // [T*8] canonical row -> slot id (first S entries valid)
     int* row_token;      // [row_cap] padded row -> token (valid rows only)
+    // small batches only (route_permute_kernel), for the kernel that fuses both GEMMs and the combine:
+    int* tok_nlocal;     // [T] local slots of each token
+    int* ready;          // [E_loc] per-row-tile counters, zeroed here
+    int* tok_done;       // [T * done_cols] per-(token, column tile) counters, zeroed here when done_cols > 0
+    int done_cols;
 };
 
 // Bit t of mask[e] says: token t of this block routes to local expert e.  The
@@ -259,16 +264,20 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
             m.tile_rows[t0 + i] = min(TILE_M, total - i * TILE_M);
         }
     }
+    for (int i = tid; i < E_loc; i += blockDim.x) m.ready[i] = 0;
+    for (int i = tid; i < T * m.done_cols; i += blockDim.x) m.tok_done[i] = 0;
     for (int t = tid; t < T; t += blockDim.x) {
         const int4 a = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t);
         const int4 b = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t + 1);
         const int ids[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
         const int word = t >> 5, bit = t & 31;
+        int nlocal = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const int e = ids[j] - off;
             int prow = -1;
             if (e >= 0 && e < E_loc) {
+                ++nlocal;
                 const int rank = pre[e * W + word] + __popc(mask[e * W + word] & ((1u << bit) - 1u));
                 prow = s_pad[e] + rank;
                 if (prow < 0 || prow >= row_cap) {
@@ -281,6 +290,7 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
             }
             m.slot_to_row[t * 8 + j] = prow;
         }
+        m.tok_nlocal[t] = nlocal;
     }
 }
 static_assert(P_TAIL_THREADS == P_MAX_LOCAL, "the tail keeps one expert's count per thread");

@@ -17,6 +17,7 @@ enum : int {
     DEV_TIMEOUT_DRAIN = 5,     // in-flight copies did not land during abort
     DEV_BAD_ROW = 6,           // a computed row index fell outside its buffer
     DEV_BAD_TICKET = 7,        // the last-block ticket counter in the workspace was not zero at launch
+    DEV_TIMEOUT_READY = 8,     // fused kernel: the rows a GEMM2 tile reads were never announced
 };
 
 // Clocks a bounded wait spins before it gives up (about a second at 2 GHz).
@@ -81,6 +82,23 @@ __device__ __forceinline__ float ld_shared_f32(const float* p) {
     return v;
 }
 
+// Bounded wait until a counter in global memory, bumped by other CTAs after a release fence, reaches
+// `target` (acquire loads).  Returns false when it gave up.
+__device__ __forceinline__ bool wait_counter(const int* p, int target, volatile int* abort_flag, long long limit) {
+    const long long t0 = clock64();
+    for (;;) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+        if (v >= target) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > limit) return false;
+        __nanosleep(64);
+    }
+}
+// Orders this thread's earlier generic-proxy accesses (any state space) before its later asynchronous-proxy
+// ones (bulk copies) and vice versa.
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
 // ---- TMA ------------------------------------------------------------------
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
@@ -119,6 +137,15 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
+__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+// Arrive on `bar` once every cp.async this thread has issued so far has landed (the barrier's expected count
+// must include this arrival).  Nothing blocks: the arrival is triggered by the copies' completion.
+__device__ __forceinline__ void cp_async_arrive_noinc(uint32_t bar) {
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {

@@ -322,3 +322,63 @@ def test_from_hidden_benchmark_shapes(cuda_device, cfg, n_sample):
     wl = syn.CONFIGS[cfg]
     S = _from_hidden_case(wl, cuda_device, sample_tokens=_sample(wl.tokens, n_sample, cfg))
     assert S > 0
+
+
+# ---- batches of at most 32 tokens: gather, both GEMMs and the combine as one kernel -------------------------
+@pytest.mark.parametrize("tokens,kw", [(1, {}), (5, {}), (16, {"local_expert_offset": 64}), (32, {}),
+                                       (23, {"skew": True})])
+def test_fused_small_batch_kernel_is_bit_identical_to_the_separate_kernels(cuda_device, tokens, kw):
+    wl = _wl(tokens, seed=80 + tokens, **kw)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device)
+    eng.set_small_batch_fusion(False)
+    want = eng.forward(inp).clone()
+    n_sep = eng.last_launch_count()
+    eng.set_small_batch_fusion(True)
+    got = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert eng.status() == 0
+    assert eng.last_launch_count() == 2 and n_sep == 5
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    run_and_compare(wl, cuda_device, inp=inp, eng=eng)
+    eng.close()
+
+
+def test_fused_small_batch_kernel_transposed_scales_and_full_size_layer(cuda_device):
+    wl = _wl(19, seed=90)
+    inp = syn.make_inputs(wl, cuda_device)
+    run_and_compare(wl, cuda_device, inp=dict(inp, hidden_scale=inp["hidden_scale"].t().contiguous()), hidden_scale_layout=1)
+    base = syn.CONFIGS[0]
+    for tokens in (1, 16, 32):
+        wl = syn.Workload(f"dsv3_T{tokens}_E32", tokens, base.dims, base.seed + tokens)
+        inp = syn.make_inputs(wl, cuda_device)
+        eng = make_engine(wl, cuda_device)
+        eng.set_small_batch_fusion(False)
+        want = eng.forward(inp).clone()
+        eng.set_small_batch_fusion(True)
+        for _ in range(3):  # counters left by one forward must not disturb the next
+            got = eng.forward(inp).clone()
+        torch.cuda.synchronize()
+        assert eng.status() == 0
+        assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+        run_and_compare(wl, cuda_device, inp=inp, eng=eng)
+        eng.close()
+
+
+def test_a_wait_that_runs_out_in_the_fused_small_batch_kernel(cuda_device):
+    wl = _wl(16, seed=43)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device)
+    want = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert eng.status() == 0 and eng.last_launch_count() == 2
+    eng.debug_set_fault(skip_iteration=1, wait_clocks=1 << 20)
+    eng.forward(inp)
+    torch.cuda.synchronize()
+    assert eng.status() in (1, 2, 3, 4, 5, 8), f"expected a time-out code, got {eng.status()}"
+    eng.debug_set_fault(-1, 0)
+    got = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert eng.status() == 0
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    eng.close()
