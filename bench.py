@@ -44,8 +44,8 @@ HBM_DATASHEET_GBS = 8000.0
 # traffic is scaled to a full launch by the algorithmic bytes, since both grow with the experts and rows.
 NCU_TRAFFIC_RATIO = {
     ("hbm", "gemm1_swiglu_quant"): 1.035, ("hbm", "gemm2"): 1.02,
-    ("tensor", "gemm1_swiglu_quant"): 1.14, ("tensor", "gemm2"): 1.10,
-    ("hbm", "fused_small"): 1.03,
+    ("tensor", "gemm1_swiglu_quant"): 1.31, ("tensor", "gemm2"): 0.99,
+    ("hbm", "fused_small"): 1.00,
 }
 METRIC = "fused FP8 MoE forward throughput (tokens/s; TFLOPS and roofline fraction alongside)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
