@@ -382,3 +382,20 @@ def test_a_wait_that_runs_out_in_the_fused_small_batch_kernel(cuda_device):
     assert eng.status() == 0
     assert torch.equal(got.view(torch.int16), want.view(torch.int16))
     eng.close()
+
+
+def test_every_token_count_of_the_bench_sweep(cuda_device):
+    # the token counts bench.py times on the 32-local-expert layer (the paper's three batch-size regimes), one
+    # set of weights: routing and permutation on all tokens, the output on up to 48 sampled tokens each
+    import bench
+    base = syn.CONFIGS[1]
+    ts = sorted(bench.SWEEP_TOKENS)
+    big = syn.Workload("sweep", ts[-1], base.dims, base.seed)
+    inp = syn.make_inputs(big, cuda_device)
+    eng = make_engine(big, cuda_device, poison=False)
+    for t in ts:
+        wl = syn.Workload(f"dsv3_T{t}_E32", t, base.dims, base.seed)
+        sub = {k: (v[:t] if k in ("hidden_fp8", "hidden_scale", "router_logits") else v) for k, v in inp.items()}
+        st = run_and_compare(wl, cuda_device, inp=sub, sample_tokens=_sample(t, 48, t), check_rows=False, eng=eng)
+        assert st["frac"] >= 0.995
+    eng.close()
