@@ -112,6 +112,23 @@ int moe_fp8_forward_host(moe_fp8_handle_t h, int T, const void* host_hidden_fp8,
                          float scaling_factor, void* host_out, void* stream);
 
 /*
+ * moe_fp8_forward_host for a sequence of steps: the call returns as soon as everything is enqueued.  The
+ * host-to-device copies of the step run on a copy stream of the library, the forward on `stream`, the copy of
+ * `out` back to host_out on a second copy stream, chained by events; two staging sets in the workspace
+ * alternate, so the copies of one step overlap the forward of its neighbours.  host_* buffers must be pinned
+ * (page-locked) for the copies to be asynchronous, must not be touched until moe_fp8_host_sync (or a later
+ * cudaStreamSynchronize of `stream` followed by moe_fp8_host_sync) returns, and host_out of step i may be reused
+ * from step i + 2 on only after such a wait.  The first call creates the two streams and six events (host
+ * objects; no device memory is allocated).  Results are those of moe_fp8_forward_host, bit for bit.
+ */
+int moe_fp8_forward_host_async(moe_fp8_handle_t h, int T, const void* host_hidden_fp8, const float* host_hidden_scale,
+                               const float* host_router_logits, const void* routing_bias, const void* w13,
+                               const float* w13_scale, const void* w2, const float* w2_scale, int local_expert_offset,
+                               float scaling_factor, void* host_out, void* stream);
+/* Waits until every copy enqueued by moe_fp8_forward_host_async on this handle has finished. */
+int moe_fp8_host_sync(moe_fp8_handle_t h);
+
+/*
  * The same pass started from bf16 hidden states: stage 1 of the Fused MoE description begins with "routing
  * scores via a lightweight linear projection", and the FP8 activations with their 128-wide scales are the
  * quantisation of those hidden states.  This entry computes

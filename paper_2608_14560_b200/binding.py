@@ -19,7 +19,7 @@ EXPORTS = (
     "moe_fp8_strerror", "moe_fp8_set_stage_timing", "moe_fp8_num_stages", "moe_fp8_stage_name",
     "moe_fp8_get_stage_times", "moe_fp8_expert_histogram_static", "moe_fp8_debug_set_fault",
     "moe_fp8_debug_sigmoid", "moe_fp8_forward_from_hidden", "moe_fp8_debug_export_inputs",
-    "moe_fp8_set_small_batch_fusion",
+    "moe_fp8_set_small_batch_fusion", "moe_fp8_forward_host_async", "moe_fp8_host_sync",
 )
 
 
@@ -60,6 +60,10 @@ def load_library() -> C.CDLL:
         lib.moe_fp8_forward.restype = C.c_int
         lib.moe_fp8_forward_host.argtypes = fwd
         lib.moe_fp8_forward_host.restype = C.c_int
+        lib.moe_fp8_forward_host_async.argtypes = fwd
+        lib.moe_fp8_forward_host_async.restype = C.c_int
+        lib.moe_fp8_host_sync.argtypes = [vp]
+        lib.moe_fp8_host_sync.restype = C.c_int
         lib.moe_fp8_forward_from_hidden.argtypes = [vp, C.c_int, vp, vp, vp, vp, fp, vp, fp, C.c_int, C.c_float, vp, vp]
         lib.moe_fp8_forward_from_hidden.restype = C.c_int
         lib.moe_fp8_debug_export_inputs.argtypes = [vp, C.c_int, fp, vp, fp, vp]
@@ -230,6 +234,21 @@ class MoeFp8:
     def debug_set_fault(self, skip_iteration: int = -1, wait_clocks: int = 0):
         """moe_fp8_debug_set_fault (test hook of the bounded-wait failure path)."""
         self._check(self.lib.moe_fp8_debug_set_fault(self.handle, int(skip_iteration), int(wait_clocks)))
+
+    def forward_host_async(self, host_act: dict, weights: dict, host_out: torch.Tensor, stream=None) -> torch.Tensor:
+        """moe_fp8_forward_host_async: as forward_host, but returns once the step is enqueued; call host_sync()
+        before reading host_out."""
+        T = host_act["router_logits"].shape[0]
+        self._check(self.lib.moe_fp8_forward_host_async(
+            self.handle, T, _ptr(host_act["hidden_fp8"]), _ptr(host_act["hidden_scale"]),
+            _ptr(host_act["router_logits"]), _ptr(weights["routing_bias"]), _ptr(weights["w13"]),
+            _ptr(weights["w13_scale"]), _ptr(weights["w2"]), _ptr(weights["w2_scale"]),
+            int(weights["local_expert_offset"]), float(weights["scaling_factor"]), _ptr(host_out),
+            self._stream(stream)))
+        return host_out
+
+    def host_sync(self):
+        self._check(self.lib.moe_fp8_host_sync(self.handle))
 
     def set_stage_timing(self, enable: bool):
         self._check(self.lib.moe_fp8_set_stage_timing(self.handle, int(enable)))

@@ -31,7 +31,7 @@ inline size_t align_up(size_t x, size_t a = WS_ALIGN) { return (x + a - 1) / a *
 struct WsLayout {
     size_t topk_idx, topk_w, block_hist, expert_count, expert_offset, padded_offset, tile_expert, tile_rows,
         num_m_tiles, slot_to_row, row_to_slot, row_token, tok_nlocal, ready, tok_done, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
-        stage_scale, stage_logits, stage_out, total;
+        stage_scale, stage_logits, stage_out, stage2_hidden, stage2_scale, stage2_logits, stage2_out, total;
     int row_cap, max_m_tiles, max_blocks;
 };
 
@@ -75,6 +75,11 @@ WsLayout make_layout(const moe_fp8_config& c) {
     L.stage_scale = take(Tm * (H / 128) * 4);
     L.stage_logits = take(Tm * 256 * 4);
     L.stage_out = take(Tm * H * 2);
+    // second staging set: moe_fp8_forward_host_async alternates between the two
+    L.stage2_hidden = take(Tm * H);
+    L.stage2_scale = take(Tm * (H / 128) * 4);
+    L.stage2_logits = take(Tm * 256 * 4);
+    L.stage2_out = take(Tm * H * 2);
     L.total = o;
     return L;
 }
@@ -101,7 +106,12 @@ struct moe_fp8_handle_s {
     int fault_skip_it;         // test hook, see moe_fp8_debug_set_fault
     long long fault_wait_limit;
     cudaEvent_t ev[NUM_STAGES_MAX + 1];
-    bool small_fusion;         // batches of at most F_MAX_TOKENS tokens take the single fused kernel
+    bool small_fusion;
+    // moe_fp8_forward_host_async: copy streams and the events that order the two staging sets
+    bool pipe_ready;
+    unsigned pipe_calls;
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev_in[2], ev_compute[2], ev_out[2];         // batches of at most F_MAX_TOKENS tokens take the single fused kernel
 };
 
 namespace {
@@ -274,6 +284,17 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
 int moe_fp8_destroy(moe_fp8_handle_t h) {
     if (!h) return MOE_FP8_ERR_BAD_ARG;
     moe_fp8_set_stage_timing(h, 0);
+    if (h->pipe_ready) {
+        cudaStreamSynchronize(h->s_in);
+        cudaStreamSynchronize(h->s_out);
+        for (int k = 0; k < 2; ++k) {
+            cudaEventDestroy(h->ev_in[k]);
+            cudaEventDestroy(h->ev_compute[k]);
+            cudaEventDestroy(h->ev_out[k]);
+        }
+        cudaStreamDestroy(h->s_in);
+        cudaStreamDestroy(h->s_out);
+    }
     delete h;
     return MOE_FP8_OK;
 }
@@ -635,6 +656,74 @@ int moe_fp8_debug_export_inputs(moe_fp8_handle_t h, int T, float* router_logits,
     copy(hidden_fp8, h->L.stage_hidden, Tz * H);
     copy(hidden_scale, h->L.stage_scale, Tz * (H / 128) * 4);
     if (e != cudaSuccess) return cuda_fail(h, e);
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_forward_host_async(moe_fp8_handle_t h, int T, const void* host_hidden_fp8, const float* host_hidden_scale,
+                               const float* host_router_logits, const void* routing_bias, const void* w13,
+                               const float* w13_scale, const void* w2, const float* w2_scale, int local_expert_offset,
+                               float scaling_factor, void* host_out, void* stream_v) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    if (T < 0 || T > h->cfg.max_tokens) return MOE_FP8_ERR_BAD_ARG;
+    if (T > 0 && (!host_hidden_fp8 || !host_hidden_scale || !host_router_logits || !host_out))
+        return MOE_FP8_ERR_BAD_ARG;
+    if (!h->ws) return MOE_FP8_ERR_NO_WORKSPACE;
+    if (T == 0) return MOE_FP8_OK;
+    cudaError_t e;
+    if (!h->pipe_ready) {  // first use: two copy streams and six events (host-side objects, no device memory)
+        if ((e = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(h, e);
+        if ((e = cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking)) != cudaSuccess) {
+            cudaStreamDestroy(h->s_in);
+            return cuda_fail(h, e);
+        }
+        for (int k = 0; k < 2; ++k) {
+            cudaEventCreateWithFlags(&h->ev_in[k], cudaEventDisableTiming);
+            cudaEventCreateWithFlags(&h->ev_compute[k], cudaEventDisableTiming);
+            cudaEventCreateWithFlags(&h->ev_out[k], cudaEventDisableTiming);
+        }
+        if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(h, e);
+        h->pipe_calls = 0;
+        h->pipe_ready = true;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    const int k = h->pipe_calls & 1;
+    const bool used_before = h->pipe_calls >= 2;  // this staging set has a call two steps back still to respect
+    const size_t H = h->cfg.hidden, Tz = T;
+    uint8_t* d_hidden = at<uint8_t>(h, k ? h->L.stage2_hidden : h->L.stage_hidden);
+    float* d_scale = at<float>(h, k ? h->L.stage2_scale : h->L.stage_scale);
+    float* d_logits = at<float>(h, k ? h->L.stage2_logits : h->L.stage_logits);
+    void* d_out = at<uint8_t>(h, k ? h->L.stage2_out : h->L.stage_out);
+    // inputs: after the forward that last read this staging set
+    if (used_before && (e = cudaStreamWaitEvent(h->s_in, h->ev_compute[k], 0)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMemcpyAsync(d_hidden, host_hidden_fp8, Tz * H, cudaMemcpyHostToDevice, h->s_in)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(d_scale, host_hidden_scale, Tz * (H / 128) * 4, cudaMemcpyHostToDevice, h->s_in)) !=
+            cudaSuccess ||
+        (e = cudaMemcpyAsync(d_logits, host_router_logits, Tz * 256 * 4, cudaMemcpyHostToDevice, h->s_in)) !=
+            cudaSuccess ||
+        (e = cudaEventRecord(h->ev_in[k], h->s_in)) != cudaSuccess)
+        return cuda_fail(h, e);
+    // forward: after its inputs have arrived and after the copy-out that last read this set's output area
+    if ((e = cudaStreamWaitEvent(stream, h->ev_in[k], 0)) != cudaSuccess) return cuda_fail(h, e);
+    if (used_before && (e = cudaStreamWaitEvent(stream, h->ev_out[k], 0)) != cudaSuccess) return cuda_fail(h, e);
+    const int rc = moe_fp8_forward(h, T, d_hidden, d_scale, d_logits, routing_bias, w13, w13_scale, w2, w2_scale,
+                                   local_expert_offset, scaling_factor, d_out, stream_v);
+    if (rc != MOE_FP8_OK) return rc;
+    if ((e = cudaEventRecord(h->ev_compute[k], stream)) != cudaSuccess) return cuda_fail(h, e);
+    // output: after the forward
+    if ((e = cudaStreamWaitEvent(h->s_out, h->ev_compute[k], 0)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(host_out, d_out, Tz * H * 2, cudaMemcpyDeviceToHost, h->s_out)) != cudaSuccess ||
+        (e = cudaEventRecord(h->ev_out[k], h->s_out)) != cudaSuccess)
+        return cuda_fail(h, e);
+    ++h->pipe_calls;
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_host_sync(moe_fp8_handle_t h) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    if (!h->pipe_ready) return MOE_FP8_OK;
+    cudaError_t e;
+    if ((e = cudaStreamSynchronize(h->s_in)) != cudaSuccess || (e = cudaStreamSynchronize(h->s_out)) != cudaSuccess)
+        return cuda_fail(h, e);
     return MOE_FP8_OK;
 }
 
