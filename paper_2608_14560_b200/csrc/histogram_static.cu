@@ -8,10 +8,12 @@
 
 #include <mutex>
 
+#include "limits.cuh"
+
 namespace {
 
-constexpr int P_TOKENS_PER_BLOCK = 256;  // tokens per block of the counting kernel
-constexpr int P_MAX_LOCAL = 256;         // most local experts supported
+using moe::P_MAX_LOCAL;
+using moe::P_TOKENS_PER_BLOCK;
 
 constexpr int STATIC_MAX_BLOCKS =
     (MOE_FP8_STATIC_HISTOGRAM_MAX_TOKENS + P_TOKENS_PER_BLOCK - 1) / P_TOKENS_PER_BLOCK;

@@ -10,13 +10,12 @@
 #pragma once
 #include <stdint.h>
 
+#include "limits.cuh"
 #include "ptx.cuh"
 #include "routing.cuh"
 
 namespace moe {
 
-constexpr int P_TOKENS_PER_BLOCK = 256;  // tokens handled by one block of the count/place kernels
-constexpr int P_MAX_LOCAL = 256;         // most local experts supported
 constexpr int TILE_M = 128;              // GEMM tile height (rows)
 
 struct PermuteMeta {

@@ -68,3 +68,15 @@ def test_create_rejects_bad_shapes_before_touching_the_device(field, value, rc):
 def test_no_device_means_loud_failure_not_a_fallback():
     with pytest.raises(binding.MoeFp8Error):
         binding.MoeFp8(device="cpu")
+
+
+def test_binding_constants_agree_with_the_header():
+    import re
+    from paper_2608_14560_b200 import binding
+    text = open(os.path.join(ROOT, "include", "moe_fp8.h")).read()
+    defs = {m.group(1): int(m.group(2).strip("()")) for m in re.finditer(r"#define (MOE_FP8_\w+) (\(?-?\d+\)?)", text)}
+    assert defs["MOE_FP8_STATIC_HISTOGRAM_MAX_TOKENS"] == binding.STATIC_HISTOGRAM_MAX_TOKENS
+    assert defs["MOE_FP8_ERR_STATIC_LIMIT"] == binding.ERR_STATIC_LIMIT
+    assert (defs["MOE_FP8_ERR_BAD_ARG"], defs["MOE_FP8_ERR_UNSUPPORTED_DIMS"], defs["MOE_FP8_ERR_NO_WORKSPACE"],
+            defs["MOE_FP8_ERR_CUDA"], defs["MOE_FP8_ERR_ARCH"]) == (
+        binding.ERR_BAD_ARG, binding.ERR_UNSUPPORTED_DIMS, binding.ERR_NO_WORKSPACE, binding.ERR_CUDA, binding.ERR_ARCH)
