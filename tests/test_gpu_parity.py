@@ -420,3 +420,11 @@ def test_pipelined_host_entry_point_matches_device_entry_point(cuda_device):
     for i in range(5):
         assert torch.equal(host_outs[i].view(torch.int16), want[i % 3].view(torch.int16)), f"step {i}"
     eng.close()
+
+
+def test_a_batch_of_65536_tokens(cuda_device):
+    # four times the largest benchmark batch: 528 352 padded rows, byte offsets beyond 2^32 in every row buffer
+    base = syn.CONFIGS[1]
+    wl = syn.Workload("dsv3_T65536_E32", 65536, base.dims, seed=65)
+    st = run_and_compare(wl, cuda_device, sample_tokens=_sample(65536, 96, 65), check_rows="tiles", poison=False)
+    assert st["S"] > 30000
