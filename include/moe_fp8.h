@@ -175,10 +175,14 @@ int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w
 
 /*
  * Batches of at most 32 tokens run the gather of stage 2, both GEMMs of stage 3 and the combine of stage 4 as
- * ONE kernel behind the routing kernel (the paper's short regime, T = 1-16, is bounded by routing and launch
- * overhead, and it names fusing the scatter into GEMM2's epilogue as the next step; in that kernel the CTA that
- * stores the last local row of a token sums the token's rows in routing order, so results stay bit-identical
- * to the separate kernels).  On by default; enable = 0 makes such batches take the separate kernels too.
+ * ONE kernel (the paper's short regime, T = 1-16, is bounded by routing and launch overhead, and it names
+ * fusing the scatter into GEMM2's epilogue as the next step; in that kernel the CTA that stores the last local
+ * row of a token sums the token's rows in routing order, so results stay bit-identical to the separate
+ * kernels).  Up to 16 tokens that kernel also does stages 1 and 2 -- every CTA routes and permutes the whole
+ * batch for itself and all write the same tables -- so a forward is a single launch; from 17 to 32 tokens a
+ * routing kernel runs in front of it.  The kernel's cross-CTA counters live in the workspace in two sets: a call
+ * uses one and zeroes the other, so a call that gave up on a bounded wait does not disturb later ones.
+ * On by default; enable = 0 makes such batches take the separate kernels too.
  */
 int moe_fp8_set_small_batch_fusion(moe_fp8_handle_t h, int enable);
 

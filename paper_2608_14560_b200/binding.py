@@ -228,7 +228,8 @@ class MoeFp8:
         return host_out
 
     def set_small_batch_fusion(self, enable: bool):
-        """moe_fp8_set_small_batch_fusion: batches of <= 32 tokens as one fused kernel (default) or as separate ones."""
+        """moe_fp8_set_small_batch_fusion: batches of <= 32 tokens as one fused kernel (default; a single launch per forward
+        up to 16 tokens) or as separate ones."""
         self._check(self.lib.moe_fp8_set_small_batch_fusion(self.handle, int(enable)))
 
     def debug_set_fault(self, skip_iteration: int = -1, wait_clocks: int = 0):

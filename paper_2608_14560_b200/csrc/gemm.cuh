@@ -34,10 +34,15 @@
 //               the one-per-SM grid are resident, so the counter always arrives).  The CTA that completes the
 //               last local row of a token for a column tile -- found with a per-(token, column tile)
 //               counter, nobody waits -- sums that token's rows in routing order and writes the bf16 output.
+//               Up to F_ROUTE_MAX_TOKENS tokens the kernel starts with stages 1 and 2 as well: every CTA routes
+//               and permutes the whole batch for itself (route_permute_in_cta) and all of them write the same
+//               tables, so the forward is one launch and still no CTA waits for a table.  The counters come
+//               in two sets; CTA 0 zeroes the set of the next call.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
 
+#include "permute.cuh"
 #include "ptx.cuh"
 
 namespace moe {
@@ -85,6 +90,12 @@ using GeomFull = Geometry<4, TILE_M, 8, G_EPI_WARPS * G_STORE_WARP_BYTES>;
 using GeomSmall = Geometry<6, 32, 16, 2 * G_STORE_WARP_BYTES>;
 
 constexpr int F_MAX_TOKENS = GeomSmall::A_ROWS;   // largest batch of fused_small_kernel
+// Largest batch whose routing and permutation run inside fused_small_kernel, by every CTA for itself (one token
+// per warp and round).  Measured against a routing kernel in front: 4-6 us faster per forward up to 13 tokens,
+// equal at 20, 1-6 us slower from 24 tokens up, where a CTA needs two to three rounds.
+constexpr int F_ROUTE_MAX_TOKENS = 16;
+static_assert(F_ROUTE_MAX_TOKENS <= RP_CTA_MAX_TOKENS && F_MAX_TOKENS <= RP_CTA_MAX_TOKENS, "capacity of route_permute_in_cta");
+static_assert(RP_CTA_SCRATCH_INTS * 4 <= GeomSmall::STAGE_BYTES, "the routing scratch lives in the first pipeline stage");
 
 struct GemmArgs {
     int num_kb;               // K / 128
@@ -118,6 +129,16 @@ struct FusedArgs {
     int* ready;                   // [row tiles] GEMM1 column tiles stored, zero at launch
     int* tok_done;                // [T, H/256] GEMM2 rows stored per (token, column tile), zero at launch
     __nv_bfloat16* out;           // bf16 [T, H]
+    // Routing and permutation inside the kernel (route != 0): every CTA computes stages 1 and 2 for itself.
+    int route, E_loc, expert_offset, row_cap;
+    const float* logits;          // [T, 256]
+    const __nv_bfloat16* bias;    // [256]
+    float scaling;
+    int* topk_idx;                // [T*8] out
+    float* topk_w_out;            // [T*8] out (the same buffer as topk_w)
+    PermuteMeta meta;
+    int* counters_next;           // the counter set of the NEXT fused call, zeroed by CTA 0 of this one
+    int num_counters;
 };
 
 struct GemmCtrl {
@@ -726,6 +747,18 @@ fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_consta
     pdl_wait();
     c.tmem_base = *reinterpret_cast<volatile uint32_t*>(&c.ctrl->tmem_slot);
     c.limit = g1.wait_limit;
+
+    // The previous fused call has ended (stream order), so the counters it used can be zeroed for the call
+    // after this one.
+    if (blockIdx.x == 0)
+        for (int i = threadIdx.x; i < f.num_counters; i += blockDim.x) f.counters_next[i] = 0;
+    if (f.route) {
+        // Stages 1 and 2, by every CTA for itself, in the not yet used pipeline stages.
+        if (blockIdx.x == 0 && threadIdx.x == 0) *g1.status = DEV_OK;  // first kernel of a forward: clear the fault word
+        int* scratch = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+        route_permute_in_cta(scratch, f.T, f.E_loc, f.expert_offset, f.row_cap, f.logits, f.bias, f.scaling, f.topk_idx,
+                             f.topk_w_out, f.meta, g1.status);
+    }
 
     // tokens without a local expert: their output rows are zeros, written here by the CTAs in turn
     for (int t = blockIdx.x; t < f.T; t += gridDim.x)

@@ -30,7 +30,7 @@ inline size_t align_up(size_t x, size_t a = WS_ALIGN) { return (x + a - 1) / a *
 
 struct WsLayout {
     size_t topk_idx, topk_w, block_hist, expert_count, expert_offset, padded_offset, tile_expert, tile_rows,
-        num_m_tiles, slot_to_row, row_to_slot, row_token, tok_nlocal, ready, tok_done, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
+        num_m_tiles, slot_to_row, row_to_slot, row_token, tok_nlocal, counters, num_counters, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
         stage_scale, stage_logits, stage_out, stage2_hidden, stage2_scale, stage2_logits, stage2_out, total;
     int row_cap, max_m_tiles, max_blocks;
 };
@@ -63,8 +63,10 @@ WsLayout make_layout(const moe_fp8_config& c) {
     L.row_to_slot = take(slots * 4);
     L.row_token = take(rc * 4);
     L.tok_nlocal = take(Tm * 4);
-    L.ready = take(std::max<size_t>(EL, 1) * 4);
-    L.tok_done = take(static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N) * 4);
+    // two sets of the fused small-batch kernel's counters (per row tile, per (token, column tile)): a call uses
+    // one and zeroes the other for the next call
+    L.num_counters = std::max<size_t>(EL, 1) + static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N);
+    L.counters = take(2 * L.num_counters * 4);
     L.status = take(8);  // device status word, then the ticket counter of route_permute_kernel
     L.a1 = take(rc * H);
     L.a1_scale_t = take(rc * (H / 128) * 4);
@@ -107,6 +109,7 @@ struct moe_fp8_handle_s {
     long long fault_wait_limit;
     cudaEvent_t ev[NUM_STAGES_MAX + 1];
     bool small_fusion;
+    unsigned long long fused_calls;
     // moe_fp8_forward_host_async: copy streams and the events that order the two staging sets
     bool pipe_ready;
     unsigned pipe_calls;
@@ -171,9 +174,6 @@ PermuteMeta meta_of(moe_fp8_handle_t h) {
     m.row_to_slot = at<int>(h, h->L.row_to_slot);
     m.row_token = at<int>(h, h->L.row_token);
     m.tok_nlocal = at<int>(h, h->L.tok_nlocal);
-    m.ready = at<int>(h, h->L.ready);
-    m.tok_done = at<int>(h, h->L.tok_done);
-    m.done_cols = 0;
     return m;
 }
 
@@ -274,6 +274,7 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     h->L = make_layout(*cfg);
     h->sm_count = sms;
     h->small_fusion = true;
+    h->fused_calls = 0;
     h->fault_skip_it = -1;
     h->fault_wait_limit = WAIT_LIMIT_CLOCKS;
     h->encode = reinterpret_cast<EncodeTiledFn>(fn);
@@ -308,7 +309,9 @@ int moe_fp8_set_workspace(moe_fp8_handle_t h, void* ws, size_t bytes) {
     // memory is asynchronous to the host and a forward may follow on a non-blocking stream, which does not
     // order itself behind the default stream: wait for it here.
     cudaError_t e = cudaMemset(static_cast<uint8_t*>(ws) + h->L.status, 0, 2 * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(static_cast<uint8_t*>(ws) + h->L.counters, 0, 2 * h->L.num_counters * sizeof(int));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    h->fused_calls = 0;
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->ws = static_cast<uint8_t*>(ws);
     h->ws_bytes = bytes;
@@ -393,10 +396,24 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     } while (0)
     h->stage_times_valid = false;
     mark();
+    // Batches of at most F_MAX_TOKENS tokens: gather, both GEMMs and the combine in one kernel; up to
+    // F_ROUTE_MAX_TOKENS that kernel also routes and permutes (every CTA for itself: one launch per forward).
     const bool fused = h->small_fusion && T <= F_MAX_TOKENS;
-    if (fused) m.done_cols = H / G_TILE_N;
+    const bool route_in_fused = fused && T <= F_ROUTE_MAX_TOKENS;
+    int *counters = nullptr, *counters_next = nullptr;
+    if (fused) {
+        // this call's counter set is zero: the fused call before it zeroed it (set_workspace for the first two)
+        const size_t set = h->fused_calls++ & 1;
+        counters = at<int>(h, h->L.counters) + set * h->L.num_counters;
+        counters_next = at<int>(h, h->L.counters) + (set ^ 1) * h->L.num_counters;
+    }
 
-    if (T <= P_TAIL_MAX_TOKENS) {  // routing in parallel blocks, the last one to finish does stage 2
+    if (route_in_fused) {
+        mark();
+        mark();
+        mark();
+        mark();
+    } else if (T <= P_TAIL_MAX_TOKENS) {  // routing in parallel blocks, the last one to finish does stage 2
         const int grid = min((T + 7) / 8, h->sm_count * 8);
         MOE_LAUNCH(route_permute_kernel, grid, P_TAIL_THREADS, route_permute_smem_bytes(T, EL), stream, false, T, EL,
                    local_expert_offset, row_cap, router_logits, static_cast<const __nv_bfloat16*>(routing_bias),
@@ -471,9 +488,21 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         f.slot_to_row = m.slot_to_row;
         f.topk_w = topk_w;
         f.tok_nlocal = m.tok_nlocal;
-        f.ready = m.ready;
-        f.tok_done = m.tok_done;
+        f.ready = counters;
+        f.tok_done = counters + std::max(EL, 1);
         f.out = static_cast<__nv_bfloat16*>(out);
+        f.route = route_in_fused;
+        f.E_loc = EL;
+        f.expert_offset = local_expert_offset;
+        f.row_cap = row_cap;
+        f.logits = router_logits;
+        f.bias = static_cast<const __nv_bfloat16*>(routing_bias);
+        f.scaling = scaling_factor;
+        f.topk_idx = topk_idx;
+        f.topk_w_out = topk_w;
+        f.meta = m;
+        f.counters_next = counters_next;
+        f.num_counters = static_cast<int>(h->L.num_counters);
         mark();  // gather_rows
         mark();  // gemm1
         mark();  // gemm2

@@ -29,11 +29,7 @@ struct PermuteMeta {
     int* slot_to_row;    // [T*8] padded row of each slot, -1 when the slot's expert is not local
     int* row_to_slot;    // [T*8] canonical row -> slot id (first S entries valid)
     int* row_token;      // [row_cap] padded row -> token (valid rows only)
-    // small batches only (route_permute_kernel), for the kernel that fuses both GEMMs and the combine:
-    int* tok_nlocal;     // [T] local slots of each token
-    int* ready;          // [E_loc] per-row-tile counters, zeroed here
-    int* tok_done;       // [T * done_cols] per-(token, column tile) counters, zeroed here when done_cols > 0
-    int done_cols;
+    int* tok_nlocal;     // [T] local slots of each token (small batches only: route_permute_kernel / _in_cta)
 };
 
 // Bit t of mask[e] says: token t of this block routes to local expert e.  The
@@ -263,8 +259,6 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
             m.tile_rows[t0 + i] = min(TILE_M, total - i * TILE_M);
         }
     }
-    for (int i = tid; i < E_loc; i += blockDim.x) m.ready[i] = 0;
-    for (int i = tid; i < T * m.done_cols; i += blockDim.x) m.tok_done[i] = 0;
     for (int t = tid; t < T; t += blockDim.x) {
         const int4 a = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t);
         const int4 b = __ldcg(reinterpret_cast<const int4*>(topk_idx) + 2 * t + 1);
@@ -293,6 +287,126 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
     }
 }
 static_assert(P_TAIL_THREADS == P_MAX_LOCAL, "the tail keeps one expert's count per thread");
+
+// Stages 1 and 2 for a batch of at most 32 tokens, computed by ONE thread block for itself: every CTA of the
+// fused small-batch kernel runs this on the same inputs and writes the same tables (to the same addresses, with
+// the same values), so no CTA ever waits for another one and no separate routing launch is needed.  Same
+// arithmetic and outputs as route_permute_kernel.  `scratch` is RP_CTA_SCRATCH_INTS ints of shared memory;
+// the block needs at least P_MAX_LOCAL threads and T warps are busy at a time.  Ends with a block barrier after
+// which every thread of the block may read the tables.
+constexpr int RP_CTA_MAX_TOKENS = 32;
+constexpr int RP_CTA_SCRATCH_INTS = RP_CTA_MAX_TOKENS * 8 + P_MAX_LOCAL + 2 * (P_MAX_LOCAL + 1);
+__device__ __forceinline__ void route_permute_in_cta(int* scratch, int T, int E_loc, int off, int row_cap,
+                                                     const float* __restrict__ logits,
+                                                     const __nv_bfloat16* __restrict__ bias, float scaling,
+                                                     int* topk_idx, float* topk_w, const PermuteMeta& m, int* status) {
+    int* s_idx = scratch;                                                  // [T][8] selected experts
+    uint32_t* mask = reinterpret_cast<uint32_t*>(scratch + RP_CTA_MAX_TOKENS * 8);   // [P_MAX_LOCAL] bit t: token t
+    int* s_cnt = scratch + RP_CTA_MAX_TOKENS * 8 + P_MAX_LOCAL;            // [P_MAX_LOCAL + 1]
+    int* s_pad = s_cnt + P_MAX_LOCAL + 1;                                  // [P_MAX_LOCAL + 1]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+    if (tid < P_MAX_LOCAL) mask[tid] = 0u;
+    {
+        float bias_f[8];
+        load_bias8(bias, lane, bias_f);
+        for (int t = warp; t < T; t += nwarps) {
+            int my_idx;
+            float my_w;
+            route_token(t, lane, logits, bias_f, scaling, my_idx, my_w);
+            if (lane < R_TOPK) {
+                s_idx[t * R_TOPK + lane] = my_idx;
+                topk_idx[t * R_TOPK + lane] = my_idx;
+                topk_w[t * R_TOPK + lane] = my_w;
+            }
+        }
+    }
+    __syncthreads();
+    if (tid < T) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int e = s_idx[tid * 8 + j] - off;
+            if (e >= 0 && e < E_loc) atomicOr(&mask[e], 1u << tid);
+        }
+    }
+    __syncthreads();
+    int total = 0;
+    if (tid < P_MAX_LOCAL) {
+        total = tid < E_loc ? __popc(mask[tid]) : 0;
+        s_cnt[tid] = total;
+        s_pad[tid] = (total + TILE_M - 1) / TILE_M * TILE_M;
+    }
+    __syncthreads();
+    if (warp == 0) {  // exclusive scans of both arrays: lane l owns entries 8l .. 8l+7
+        int c[8], q[8], sc = 0, sq = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            c[i] = s_cnt[lane * 8 + i];
+            q[i] = s_pad[lane * 8 + i];
+            sc += c[i];
+            sq += q[i];
+        }
+        int ec = sc, eq = sq;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int vc = __shfl_up_sync(0xffffffffu, ec, d), vq = __shfl_up_sync(0xffffffffu, eq, d);
+            if (lane >= d) {
+                ec += vc;
+                eq += vq;
+            }
+        }
+        int bc = ec - sc, bq = eq - sq;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            s_cnt[lane * 8 + i] = bc;
+            s_pad[lane * 8 + i] = bq;
+            bc += c[i];
+            bq += q[i];
+        }
+        if (lane == 31) {
+            s_cnt[P_MAX_LOCAL] = ec;
+            s_pad[P_MAX_LOCAL] = eq;
+        }
+    }
+    __syncthreads();
+    if (tid < E_loc) {
+        m.expert_count[tid] = total;
+        m.expert_offset[tid] = s_cnt[tid];
+        m.padded_offset[tid] = s_pad[tid];
+        const int t0 = s_pad[tid] / TILE_M;
+        for (int i = 0; i * TILE_M < total; ++i) {
+            m.tile_expert[t0 + i] = tid;
+            m.tile_rows[t0 + i] = min(TILE_M, total - i * TILE_M);
+        }
+    }
+    if (tid == 0) {  // entries past E_loc count nothing, so entry E_loc already holds the totals
+        *m.num_m_tiles = s_pad[E_loc] / TILE_M;
+        m.expert_offset[E_loc] = s_cnt[E_loc];
+        m.padded_offset[E_loc] = s_pad[E_loc];
+    }
+    if (tid < T) {
+        int nlocal = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int e = s_idx[tid * 8 + j] - off;
+            int prow = -1;
+            if (e >= 0 && e < E_loc) {
+                ++nlocal;
+                const int rank = __popc(mask[e] & ((1u << tid) - 1u));
+                prow = s_pad[e] + rank;
+                if (prow < 0 || prow >= row_cap) {
+                    atomicExch(status, DEV_BAD_ROW);
+                    prow = -1;
+                } else {
+                    m.row_to_slot[s_cnt[e] + rank] = tid * 8 + j;
+                    m.row_token[prow] = tid;
+                }
+            }
+            m.slot_to_row[tid * 8 + j] = prow;
+        }
+        m.tok_nlocal[tid] = nlocal;
+    }
+    __syncthreads();
+}
 
 // One warp per padded row: copy the token's FP8 row (K bytes) and write its
 // K/128 scales transposed ([K/128, row_cap]) so the GEMM epilogue reads them
