@@ -26,18 +26,20 @@
 // Two kernels are built from these roles:
 //   grouped_gemm_kernel<MODE>   one GEMM per launch (any batch size);
 //   fused_small_kernel          batches of at most F_MAX_TOKENS tokens: the gather of stage 2, GEMM1, GEMM2
-//               and the weighted combine of stage 4 in ONE launch.  Every CTA first works through its GEMM1
-//               tiles, then its GEMM2 tiles.  Warp 3 gathers the (few) token rows of a GEMM1 tile straight
-//               from the token-major input with cp.async.  A GEMM2 tile starts once a counter in global
-//               memory says that all GEMM1 column tiles of its row tile have been stored (bounded wait; GEMM1
-//               tiles never wait for another CTA and precede the GEMM2 tiles in every CTA, and all CTAs of
-//               the one-per-SM grid are resident, so the counter always arrives).  The CTA that completes the
-//               last local row of a token for a column tile -- found with a per-(token, column tile)
-//               counter, nobody waits -- sums that token's rows in routing order and writes the bf16 output.
-//               Up to F_ROUTE_MAX_TOKENS tokens the kernel starts with stages 1 and 2 as well: every CTA routes
-//               and permutes the whole batch for itself (route_permute_in_cta) and all of them write the same
-//               tables, so the forward is one launch and still no CTA waits for a table.  The counters come
-//               in two sets; CTA 0 zeroes the set of the next call.
+//               and the weighted combine of stage 4 in ONE launch, with the operands swapped (weights on the
+//               M side of the MMA, the tile's at most 32 token rows on the N side; see "weights on M" below).
+//               Every CTA first works through its GEMM1 tiles, then its GEMM2 tiles.  Warp 3 gathers the (few)
+//               token rows of a GEMM1 tile straight from the token-major input with cp.async.  A GEMM2 tile
+//               starts once a counter in global memory says that all GEMM1 column tiles of its row tile have
+//               been stored (bounded wait; GEMM1 tiles never wait for another CTA and precede the GEMM2 tiles
+//               in every CTA, and all CTAs of the one-per-SM grid are resident, so the counter always
+//               arrives).  The CTA that completes the last local row of a token for a column tile -- found
+//               with a per-(token, column tile) counter, nobody waits -- sums that token's rows in routing
+//               order and writes the bf16 output.  Up to F_ROUTE_MAX_TOKENS tokens the kernel starts with
+//               stages 1 and 2 as well: every CTA routes and permutes the whole batch for itself
+//               (route_permute_in_cta) and all of them write the same tables, so the forward is one launch
+//               and still no CTA waits for a table.  The counters come in two sets; CTA 0 zeroes the set of
+//               the next call.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
@@ -85,9 +87,10 @@ struct Geometry {
 };
 // one GEMM per launch: full 128-row A tiles, 4 stages of 48 KB
 using GeomFull = Geometry<4, TILE_M, 8, G_EPI_WARPS * G_STORE_WARP_BYTES>;
-// fused small-batch kernel: a row tile holds at most 32 rows, so the A slot shrinks to 4 KB and six stages fit:
-// 192 KB of weights in flight per SM instead of 128 KB, which is what a weight-streaming CTA is limited by
-using GeomSmall = Geometry<6, 32, 16, 2 * G_STORE_WARP_BYTES>;
+// fused small-batch kernel: a row tile holds at most 32 token rows, so their slot shrinks to 4 KB and six
+// stages fit: 192 KB of weights in flight per SM instead of 128 KB, which is what a weight-streaming CTA is
+// limited by; 512 bytes of output staging per epilogue warp
+using GeomSmall = Geometry<6, 32, 16, G_EPI_WARPS * 512>;
 
 constexpr int F_MAX_TOKENS = GeomSmall::A_ROWS;   // largest batch of fused_small_kernel
 // Largest batch whose routing and permutation run inside fused_small_kernel, by every CTA for itself (one token
@@ -144,7 +147,7 @@ struct FusedArgs {
 struct GemmCtrl {
     uint64_t full[G_MAX_STAGES];   // stage filled (TMA transaction bytes)
     uint64_t done[G_MAX_STAGES];   // the MMAs that read the stage have finished: stage free AND accumulator ready
-    uint64_t tmem_empty[G_ACC_BUFS];
+    uint64_t tmem_empty[G_MAX_STAGES];   // accumulator buffers: two, or one per stage (weights-on-M roles)
     uint64_t amax_bar[2];
     uint64_t drain_bar[2];
     uint64_t sync_bar[2];      // fused kernel: rendezvous of the epilogue warps at the end of a tile
@@ -200,9 +203,7 @@ __device__ __forceinline__ void gemm_cta_setup(Cta& c, uint8_t* smem_raw, int fu
             mbar_init(smem_u32(&ctrl->full[s]), full_count);
             mbar_init(smem_u32(&ctrl->done[s]), 1);
         }
-        for (int b = 0; b < G_ACC_BUFS; ++b) {
-            mbar_init(smem_u32(&ctrl->tmem_empty[b]), G_EPI_WARPS);
-        }
+        for (int b = 0; b < G_MAX_STAGES; ++b) mbar_init(smem_u32(&ctrl->tmem_empty[b]), G_EPI_WARPS);
         mbar_init(smem_u32(&ctrl->amax_bar[0]), G_EPI_WARPS * 32);
         mbar_init(smem_u32(&ctrl->amax_bar[1]), G_EPI_WARPS * 32);
         mbar_init(smem_u32(&ctrl->drain_bar[0]), 1);
@@ -219,9 +220,10 @@ __device__ __forceinline__ void gemm_cta_setup(Cta& c, uint8_t* smem_raw, int fu
 }
 
 // ---------------- TMA producer (one thread) ----------------
-// MODE 1: B tile = 4 x 64 weight rows (gate[0,64) | up[0,64) | gate[64,128) | up[64,128) of the tile's 128
-// columns); MODE 2: B tile = 2 x 128 rows.  FUSED and MODE 1: the A tile and the scales come from the gather
-// warp instead; FUSED and MODE 2: the tile's A rows are GEMM1's output and must have been stored.
+// MODE 1: weight tile = 4 x 64 weight rows (gate[0,64) | up[0,64) | gate[64,128) | up[64,128) of the tile's 128
+// columns; in the fused kernel gate[0,128) | up[0,128)); MODE 2: 2 x 128 rows.  FUSED and MODE 1: the token
+// rows and the scales come from the gather warp instead; FUSED and MODE 2: the tile's token rows are GEMM1's
+// output and must have been stored.
 template <int MODE, bool FUSED, class GEO>
 __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* tmA, const CUtensorMap* tmB,
                                                const GemmArgs& g, const FusedArgs* f, int ready_target, TileRange tr,
@@ -249,9 +251,11 @@ __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* 
             const int k0 = kb * G_BLOCK_K;
             if (MODE == 1) {
                 const int gr = wrow + g.gate_row0 + n * 128, ur = wrow + g.up_row0 + n * 128;
+                // weights on N: gate[0,64) | up[0,64) | gate[64,128) | up[64,128); on M (fused kernel):
+                // gate[0,128) | up[0,128)
                 tma_load_2d(b_dst, tmB, k0, gr, bar);
-                tma_load_2d(b_dst + G_B_BYTES / 4, tmB, k0, ur, bar);
-                tma_load_2d(b_dst + G_B_BYTES / 2, tmB, k0, gr + 64, bar);
+                tma_load_2d(b_dst + G_B_BYTES / 4, tmB, k0, FUSED ? gr + 64 : ur, bar);
+                tma_load_2d(b_dst + G_B_BYTES / 2, tmB, k0, FUSED ? ur : gr + 64, bar);
                 tma_load_2d(b_dst + 3 * G_B_BYTES / 4, tmB, k0, ur + 64, bar);
             } else {
                 const int br = wrow + n * G_TILE_N;
@@ -438,12 +442,10 @@ __device__ __forceinline__ bool epilogue_rendezvous(const Cta& c, uint32_t& n) {
 // MODE 1: gate/up projection + SwiGLU + re-quantisation; tmOut describes the e4m3 output [row_cap, I] for
 //         64-byte x 32-row TMA stores.
 // MODE 2: down projection, bf16 rows out in the tile-blocked layout.
-// FUSED:  MODE 1 announces every stored tile in f->ready; MODE 2 counts the stored rows per (token, column
-//         tile) and combines the tokens it completes.
-template <int MODE, bool FUSED, class GEO>
-__device__ __forceinline__ void epilogue_tiles(const Cta& c, const CUtensorMap* tmOut, const GemmArgs& g,
-                                               const FusedArgs* f, TileRange tr, uint32_t& it, uint32_t& tile_iter,
-                                               uint32_t& sync_iter, bool& ok) {
+template <int MODE, class GEO>
+__device__ __forceinline__ void epilogue_tiles(const Cta& c, const CUtensorMap* tmOut, const GemmArgs& g, TileRange tr,
+                                               uint32_t& it, uint32_t& tile_iter, bool& ok) {
+    static_assert(GEO::A_ROWS == TILE_M && GEO::STORE_BYTES == G_EPI_WARPS * G_STORE_WARP_BYTES, "full row tiles");
     GemmCtrl* ctrl = c.ctrl;
     const int warp = c.warp, lane = c.lane;
     const int widx = warp - 4;
@@ -453,11 +455,8 @@ __device__ __forceinline__ void epilogue_tiles(const Cta& c, const CUtensorMap* 
     const uint32_t t_lane = c.tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + half * G_HALF_N;
     const size_t row_cap = static_cast<size_t>(g.row_cap);
     float* amax_x = c.amax_x;
-    // staging of this warp's GEMM1 rows; with the small geometry only the first row quadrant ever stores
-    uint8_t* stage = c.store_stage + (GEO::STORE_BYTES == G_EPI_WARPS * G_STORE_WARP_BYTES ? widx : half) * G_STORE_WARP_BYTES;
-    // row of the scale slot this thread reads (rows that are not fetched borrow the last fetched one: their
-    // accumulator rows are never stored)
-    const int scale_row = GEO::A_ROWS == TILE_M ? r_in_tile : (r_in_tile < GEO::A_ROWS ? r_in_tile : GEO::A_ROWS - 1);
+    uint8_t* stage = c.store_stage + widx * G_STORE_WARP_BYTES;  // staging of this warp's GEMM1 rows
+    const int scale_row = r_in_tile;
     const int num_kb = g.num_kb;
     for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
         const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
@@ -573,25 +572,6 @@ __device__ __forceinline__ void epilogue_tiles(const Cta& c, const CUtensorMap* 
                 if (half == 0 && r_in_tile < rows_valid)
                     g.out_scale_t[static_cast<size_t>(n) * row_cap + row] = sc;
             }
-            if (FUSED) {
-                // Announce the tile: the rows are in global memory once the bulk stores have completed (not
-                // merely been read); every thread's writes are fenced before the epilogue warps meet, and the
-                // announcing thread fences once more behind the barrier.
-                if (lane == 0) {
-                    bulk_wait_all();
-                    fence_proxy_async();
-                }
-                __threadfence();
-                if (!epilogue_rendezvous(c, sync_iter)) {
-                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                    ok = false;
-                    break;
-                }
-                if (warp == 4 && lane == 0) {
-                    __threadfence();
-                    atomicAdd(f->ready + m_tile, 1);
-                }
-            }
         } else {
             // bf16 rows out in a tile-blocked layout: block (row tile, column tile, half, quadrant) holds
             // this warp's 32 rows x 128 columns as [8 column groups][32 rows][16 bf16], so every warp
@@ -611,60 +591,285 @@ __device__ __forceinline__ void epilogue_tiles(const Cta& c, const CUtensorMap* 
                     st_global_v8(blk + q * 1024, w);
                 }
             }
-            if (FUSED) {
-                // Stage 4 without a kernel of its own.  Once both halves of the tile are stored and fenced, the
-                // thread of each valid row bumps the counter of (its token, this column tile); whoever brings
-                // it to the token's number of local slots knows that all of the token's rows for these 256
-                // columns are in memory and sums them, in routing order, exactly as combine_kernel does.
+        }
+    }
+}
+
+// ================= weights on M: the roles of the fused small-batch kernel =================
+// With at most 32 token rows in a tile, a 128 x 256 accumulator holds 96 rows of padding, and the two
+// epilogue warps that own the 32 real rows (TMEM lanes) do all of the per-K-block promotion.  Here the
+// operands are swapped instead: the 256 weight rows of the tile are the M side (two MMAs of M = 128 per K
+// step), the 32 token rows the N side.  An accumulator is then 128 lanes x 32 columns per weight-row block,
+// 64 columns per K-block: every stage gets an accumulator buffer of its own (6 x 64 of the 512 columns),
+// so the hand-over latencies overlap six deep, and every epilogue thread owns one weight row (an output
+// column) for 16 tokens -- 32 loads and 32 FMAs per K-block instead of 128, evenly over all eight warps.
+// Element for element the arithmetic is the one of the other orientation.
+constexpr int WM_TOKENS = 32;                       // N of the MMA: token rows of a tile
+constexpr int WM_BUF_COLS = 2 * WM_TOKENS;          // TMEM columns per K-block: two weight-row blocks
+static_assert(G_MAX_STAGES * WM_BUF_COLS <= static_cast<int>(G_TMEM_COLS), "one accumulator buffer per stage");
+
+template <class GEO>
+__device__ __forceinline__ void issuer_tiles_wm(const Cta& c, const GemmArgs& g, TileRange tr, uint32_t mine,
+                                                uint32_t& it, bool& ok) {
+    static_assert(GEO::A_ROWS == WM_TOKENS, "the token slot of a stage is the MMA's N operand");
+    static_assert(GEO::SCALE_SLOTS >= 2 * GEO::STAGES + 1, "the gather may be two pipelines ahead of the epilogue");
+    GemmCtrl* ctrl = c.ctrl;
+    const uint32_t idesc = umma_idesc_f8(TILE_M, WM_TOKENS);
+    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+            if ((it & 1) != mine) continue;
+            const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
+            const uint32_t tok_addr = c.smem_base + s * GEO::STAGE_BYTES;
+            const uint64_t t_desc = umma_desc_sw128(tok_addr);
+            const uint64_t w0_desc = umma_desc_sw128(tok_addr + GEO::A_BYTES);
+            const uint64_t w1_desc = umma_desc_sw128(tok_addr + GEO::A_BYTES + G_B_BYTES / 2);
+            const uint32_t d_tmem = c.tmem_base + s * WM_BUF_COLS;
+            if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, c.abort_flag, c.limit)) {
+                raise(ctrl, g.status, DEV_TIMEOUT_MMA_SMEM);
+                ok = false;
+                break;
+            }
+            // the buffer of this stage was last used one pipeline round ago
+            if (!mbar_wait(smem_u32(&ctrl->tmem_empty[s]), ph ^ 1, c.abort_flag, c.limit)) {
+                raise(ctrl, g.status, DEV_TIMEOUT_MMA_TMEM);
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+#pragma unroll
+            for (int k = 0; k < G_BLOCK_K / 32; ++k) umma_f8(d_tmem, w0_desc + 2 * k, t_desc + 2 * k, idesc, k > 0);
+#pragma unroll
+            for (int k = 0; k < G_BLOCK_K / 32; ++k)
+                umma_f8(d_tmem + WM_TOKENS, w1_desc + 2 * k, t_desc + 2 * k, idesc, k > 0);
+            umma_commit(smem_u32(&ctrl->done[s]));
+        }
+    }
+}
+
+// MODE 1: weight-row block 0 = 128 gate rows, block 1 = the matching 128 up rows; SwiGLU, re-quantisation per
+//         token over the tile's 128 output columns, e4m3 bytes and scales out, tile announced in f->ready.
+// MODE 2: blocks 0 / 1 = output columns [0,128) / [128,256) of the tile; bf16 out in the tile-blocked layout,
+//         then the per-(token, column tile) counters and the combine of the tokens this CTA completes.
+template <int MODE, class GEO>
+__device__ __forceinline__ void epilogue_tiles_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, TileRange tr,
+                                                  uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, bool& ok) {
+    GemmCtrl* ctrl = c.ctrl;
+    const int warp = c.warp, lane = c.lane;
+    const int th = (warp - 4) >> 2;          // which 16 of the tile's 32 token rows
+    const int quad = warp & 3;               // TMEM lane quadrant this warp may read
+    // (lane l of quadrant q holds weight row 32 q + l of each 128-row block)
+    const uint32_t t_lane = c.tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + th * 16;
+    const size_t row_cap = static_cast<size_t>(g.row_cap);
+    uint32_t* amax_x = reinterpret_cast<uint32_t*>(c.amax_x);   // [2 parities][2 token halves][4 quadrants][16]
+    const int num_kb = g.num_kb;
+    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
+        const int e = __ldcg(g.tile_expert + m_tile);
+        const int rows_valid = __ldcg(g.tile_rows + m_tile);
+        const int sblocks = g.w_rows_per_expert / 128;
+        const float* ws0;  // weight-scale rows of block 0 / block 1
+        const float* ws1;
+        if (MODE == 1) {
+            ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.gate_row0 / 128 + n) * num_kb;
+            ws1 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.up_row0 / 128 + n) * num_kb;
+        } else {
+            ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + 2 * n) * num_kb;
+            ws1 = ws0 + num_kb;
+        }
+        float acc[32];  // [0,16): block 0, [16,32): block 1, for tokens 16 th .. 16 th + 15
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[j] = 0.0f;
+
+        float s0 = __ldg(ws0), s1 = __ldg(ws1);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+            const float w0 = s0, w1 = s1;
+            if (kb + 1 < num_kb) {
+                s0 = __ldg(ws0 + kb + 1);
+                s1 = __ldg(ws1 + kb + 1);
+            }
+            const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph, c.abort_flag, c.limit))) {
+                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                ok = false;
+                break;
+            }
+            tc_fence_after();
+            // the MMAs of this K-block have finished, hence its stage -- tokens, weights and scales -- had landed
+            const float4* sp = reinterpret_cast<const float4*>(c.scale_ring + (it % GEO::SCALE_SLOTS) * GEO::A_ROWS + th * 16);
+            float sa[16];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float4 x = sp[q];
+                sa[4 * q] = x.x;
+                sa[4 * q + 1] = x.y;
+                sa[4 * q + 2] = x.z;
+                sa[4 * q + 3] = x.w;
+            }
+            float v[32];
+            tmem_ld16x2(t_lane + s * WM_BUF_COLS, t_lane + s * WM_BUF_COLS + WM_TOKENS, v);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[s]));
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                acc[t] = fmaf(v[t], sa[t] * w0, acc[t]);
+                acc[16 + t] = fmaf(v[16 + t], sa[t] * w1, acc[16 + t]);
+            }
+        }
+        if (!ok) break;
+
+        const size_t row0 = static_cast<size_t>(m_tile) * TILE_M + th * 16;  // padded row of this thread's token 0
+        const int valid = min(16, rows_valid - th * 16);                     // tokens of this thread that exist
+        if (MODE == 1) {
+            float cc[16];
+            uint32_t wmax[16];
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                const float gt = acc[t];
+                cc[t] = __fdividef(gt, 1.0f + __expf(-gt)) * acc[16 + t];
+                // |x| as an integer orders like the float: the warp's maximum over its 32 output columns
+                wmax[t] = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(cc[t])));
+            }
+            const uint32_t par = tile_iter & 1;
+            uint32_t* xq = amax_x + ((par * 2 + th) * 4) * 16;
+            {
+                uint32_t mine = 0;
+#pragma unroll
+                for (int t = 0; t < 16; ++t)
+                    if (lane == t) mine = wmax[t];
+                if (lane < 16) xq[quad * 16 + lane] = mine;
+            }
+            const uint32_t xbar = smem_u32(&ctrl->amax_bar[par]);
+            mbar_arrive(xbar);
+            if (!__all_sync(0xffffffffu, mbar_wait(xbar, (tile_iter >> 1) & 1, c.abort_flag, c.limit))) {
+                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                ok = false;
+                break;
+            }
+            ++tile_iter;
+            // lane t < 16 owns the scale of token t's 128-column block; everybody fetches its reciprocal
+            float my_sc = 1.0f, my_inv = 1.0f;
+            if (lane < 16) {
+                const volatile uint32_t* xv = xq + lane;
+                const float amax = __uint_as_float(max(max(xv[0], xv[16]), max(xv[32], xv[48])));
+                my_sc = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 448.0f);
+                my_inv = __frcp_rn(my_sc);
+            }
+            // Narrow global stores are slow (a warp's 32 single bytes cost tens of clocks): the codes are
+            // transposed through this warp's 512 bytes of staging, [16 tokens][32 columns], and leave as
+            // 16-byte stores -- lane l carries 16 columns of token l / 2.
+            uint8_t* wst = c.store_stage + (warp - 4) * 512;
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                const float inv_sc = __shfl_sync(0xffffffffu, my_inv, t);
+                wst[t * 32 + lane] =
+                    static_cast<uint8_t>(__nv_cvt_float_to_fp8(cc[t] * inv_sc, __NV_SATFINITE, __NV_E4M3));
+            }
+            __syncwarp();
+            if ((lane >> 1) < valid)
+                *reinterpret_cast<uint4*>(g.out_fp8 + (row0 + (lane >> 1)) * g.out_cols + n * 128 + quad * 32 + (lane & 1) * 16) =
+                    *reinterpret_cast<const uint4*>(wst + (lane >> 1) * 32 + (lane & 1) * 16);
+            if (quad == 0 && lane < valid) g.out_scale_t[static_cast<size_t>(n) * row_cap + row0 + lane] = my_sc;
+            __syncwarp();
+            // Announce the tile: every thread's stores are fenced before the epilogue warps meet, and the
+            // announcing thread fences once more behind the barrier.  (The rows are read by other CTAs' copy
+            // engines: plain stores here, asynchronous-proxy loads there.)
+            fence_proxy_async();
+            __threadfence();
+            if (!epilogue_rendezvous(c, sync_iter)) {
+                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                ok = false;
+                break;
+            }
+            if (warp == 4 && lane == 0) {
                 __threadfence();
-                if (!epilogue_rendezvous(c, sync_iter)) {
-                    if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                    ok = false;
-                    break;
+                atomicAdd(f->ready + m_tile, 1);
+            }
+        } else {
+            // bf16 out through this warp's 512 bytes of staging, eight tokens x 32 columns at a time, so that
+            // the rows leave as 16-byte stores: lane l carries 8 columns of token l / 4 (half of a 32-byte
+            // group of the tile-blocked layout)
+            __nv_bfloat16* wst = reinterpret_cast<__nv_bfloat16*>(c.store_stage + (warp - 4) * 512);
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) wst[t * 32 + lane] = __float2bfloat16_rn(acc[j * 16 + h * 8 + t]);
+                    __syncwarp();
+                    const int t = h * 8 + (lane >> 2), ch0 = quad * 32 + (lane & 3) * 8;
+                    if (t < valid)
+                        *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(g.out_bf16) +
+                                                  y_block_offset(static_cast<int>(row0) + t, n * 16 + j * 8 + (ch0 >> 4), g.n_tiles) +
+                                                  (ch0 & 15) * 2) =
+                            *reinterpret_cast<const uint4*>(wst + (lane >> 2) * 32 + (lane & 3) * 8);
+                    __syncwarp();
                 }
-                if (half == 0) {
-                    int tok = -1;
-                    bool last = false;
-                    if (r_in_tile < rows_valid) {
-                        tok = __ldcg(f->row_token + row);
-                        __threadfence();
-                        const int before = atomicAdd(f->tok_done + static_cast<size_t>(tok) * g.n_tiles + n, 1);
-                        last = before == __ldcg(f->tok_nlocal + tok) - 1;
-                    }
-                    uint32_t todo = __ballot_sync(0xffffffffu, last);
-                    if (todo) __threadfence();
-                    while (todo) {
-                        const int src = __ffs(todo) - 1;
-                        todo &= todo - 1;
-                        const int t = __shfl_sync(0xffffffffu, tok, src);
-                        // lane l owns columns n*256 + 8 l .. + 8: half of the 32-byte group n*16 + l/2
-                        float o[8];
+            }
+            // Stage 4 without a kernel of its own.  Once the tile is stored and fenced, the thread of each valid
+            // row bumps the counter of (its token, this column tile); whoever brings it to the token's number of
+            // local slots knows that all of the token's rows for these 256 columns are in memory and sums
+            // them, in routing order, exactly as combine_kernel does.
+            __threadfence();
+            if (!epilogue_rendezvous(c, sync_iter)) {
+                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+                ok = false;
+                break;
+            }
+            {
+                // epilogue warp w looks after the rows w, w + 8, w + 16, w + 24 of the tile (lanes 0..3), so up
+                // to eight completed tokens are summed at the same time
+                int tok = -1;
+                bool last = false;
+                const int r_mine = (warp - 4) + 8 * lane;
+                if (lane < 4 && r_mine < rows_valid) {
+                    tok = __ldcg(f->row_token + static_cast<size_t>(m_tile) * TILE_M + r_mine);
+                    __threadfence();
+                    const int before = atomicAdd(f->tok_done + static_cast<size_t>(tok) * g.n_tiles + n, 1);
+                    last = before == __ldcg(f->tok_nlocal + tok) - 1;
+                }
+                uint32_t todo = __ballot_sync(0xffffffffu, last);
+                if (todo) __threadfence();
+                while (todo) {
+                    const int src = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const int t = __shfl_sync(0xffffffffu, tok, src);
+                    // lane l owns columns n*256 + 8 l .. + 8: half of the 32-byte group n*16 + l/2.  All loads
+                    // first, then the sum in routing order.
+                    const int4 ra = __ldcg(reinterpret_cast<const int4*>(f->slot_to_row) + 2 * t);
+                    const int4 rb = __ldcg(reinterpret_cast<const int4*>(f->slot_to_row) + 2 * t + 1);
+                    const float4 wa = __ldcg(reinterpret_cast<const float4*>(f->topk_w) + 2 * t);
+                    const float4 wb = __ldcg(reinterpret_cast<const float4*>(f->topk_w) + 2 * t + 1);
+                    const int rr[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+                    const float ww[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+                    uint4 u[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) o[i] = 0.0f;
+                    for (int j = 0; j < 8; ++j)
+                        if (rr[j] >= 0)
+                            u[j] = __ldcg(reinterpret_cast<const uint4*>(
+                                reinterpret_cast<const uint8_t*>(g.out_bf16) +
+                                y_block_offset(rr[j], n * 16 + (lane >> 1), g.n_tiles) + (lane & 1) * 16));
+                    float o[8];
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const int r = __ldcg(f->slot_to_row + t * 8 + j);
-                            if (r < 0) continue;
-                            const float wj = __ldcg(f->topk_w + t * 8 + j);
-                            const uint4 u = __ldcg(reinterpret_cast<const uint4*>(
-                                reinterpret_cast<const uint8_t*>(g.out_bf16) + y_block_offset(r, n * 16 + (lane >> 1), g.n_tiles) +
-                                (lane & 1) * 16));
-                            const uint32_t uu[4] = {u.x, u.y, u.z, u.w};
+                    for (int i = 0; i < 8; ++i) o[i] = 0.0f;
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                o[2 * i] = fmaf(wj, __uint_as_float(uu[i] << 16), o[2 * i]);
-                                o[2 * i + 1] = fmaf(wj, __uint_as_float(uu[i] & 0xffff0000u), o[2 * i + 1]);
-                            }
-                        }
-                        uint32_t p[4];
+                    for (int j = 0; j < 8; ++j) {
+                        if (rr[j] < 0) continue;
+                        const uint32_t uu[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            const __nv_bfloat162 pr = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
-                            p[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                            o[2 * i] = fmaf(ww[j], __uint_as_float(uu[i] << 16), o[2 * i]);
+                            o[2 * i + 1] = fmaf(ww[j], __uint_as_float(uu[i] & 0xffff0000u), o[2 * i + 1]);
                         }
-                        *reinterpret_cast<uint4*>(f->out + static_cast<size_t>(t) * f->H + n * G_TILE_N + lane * 8) =
-                            make_uint4(p[0], p[1], p[2], p[3]);
                     }
+                    uint32_t p[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const __nv_bfloat162 pr = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+                        p[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                    }
+                    *reinterpret_cast<uint4*>(f->out + static_cast<size_t>(t) * f->H + n * G_TILE_N + lane * 8) =
+                        make_uint4(p[0], p[1], p[2], p[3]);
                 }
             }
         }
@@ -710,8 +915,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
     } else {
         reg_alloc<232>();
-        uint32_t tile_iter = 0, sync_iter = 0;
-        epilogue_tiles<MODE, false, GEO>(c, &tmOut, g, nullptr, tr, it, tile_iter, sync_iter, ok);
+        uint32_t tile_iter = 0;
+        epilogue_tiles<MODE, GEO>(c, &tmOut, g, tr, it, tile_iter, ok);
         if (c.lane == 0) bulk_wait_all();
     }
 
@@ -728,8 +933,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 // two weight tensors.
 __global__ void __launch_bounds__(G_THREADS, 1)
 fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB1,
-                   const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmOut,
-                   const GemmArgs g1, const GemmArgs g2, const FusedArgs f) {
+                   const __grid_constant__ CUtensorMap tmB2, const GemmArgs g1, const GemmArgs g2, const FusedArgs f) {
     extern __shared__ uint8_t smem_raw[];
     using GEO = GeomSmall;
     Cta c;
@@ -738,7 +942,6 @@ fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_consta
         tma_prefetch_desc(&tmA2);
         tma_prefetch_desc(&tmB1);
         tma_prefetch_desc(&tmB2);
-        tma_prefetch_desc(&tmOut);
     }
     tc_fence_before();
     __syncthreads();
@@ -782,8 +985,8 @@ fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_consta
             producer_tiles<2, true, GEO>(c, &tmA2, &tmB2, g2, &f, g1.n_tiles, tr2, it, ok);
             producer_drain<GEO>(c, g1.status, it);
         } else if ((c.warp == 1 || c.warp == 2) && c.lane == 0) {
-            issuer_tiles<GEO>(c, g1, tr1, c.warp - 1, it, ok);
-            issuer_tiles<GEO>(c, g2, tr2, c.warp - 1, it, ok);
+            issuer_tiles_wm<GEO>(c, g1, tr1, c.warp - 1, it, ok);
+            issuer_tiles_wm<GEO>(c, g2, tr2, c.warp - 1, it, ok);
             issuer_drain(c, c.warp - 1, ok);
         } else if (c.warp == 3) {
             gather_tiles<GEO>(c, g1, f, tr1, it, ok);
@@ -793,9 +996,8 @@ fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_consta
     } else {
         reg_alloc<232>();
         uint32_t tile_iter = 0, sync_iter = 0;
-        epilogue_tiles<1, true, GEO>(c, &tmOut, g1, &f, tr1, it, tile_iter, sync_iter, ok);
-        epilogue_tiles<2, true, GEO>(c, &tmOut, g2, &f, tr2, it, tile_iter, sync_iter, ok);
-        if (c.lane == 0) bulk_wait_all();
+        epilogue_tiles_wm<1, GEO>(c, g1, &f, tr1, it, tile_iter, sync_iter, ok);
+        epilogue_tiles_wm<2, GEO>(c, g2, &f, tr2, it, tile_iter, sync_iter, ok);
     }
 
     tc_fence_before();

@@ -508,7 +508,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         mark();  // gemm2
         mark();  // combine
         MOE_LAUNCH(fused_small_kernel, h->sm_count, G_THREADS, GeomSmall::SMEM_BYTES, stream, pdl, h->tm_a2_small,
-                   h->tm_w13, h->tm_w2, h->tm_a2_store, g1, g2, f);
+                   h->tm_w13, h->tm_w2, g1, g2, f);
         mark();
     } else {
         {  // stage 2, continued: gather
