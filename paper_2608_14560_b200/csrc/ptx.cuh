@@ -259,6 +259,20 @@ __device__ __forceinline__ void ld_global_v8(const void* p, uint32_t (&w)[8]) {
                  : "memory");
 }
 
+// ---- packed fp32 ------------------------------------------------------------
+// Two fp32 values (bit patterns) in one 64-bit register: lo in bits 0..31.
+__device__ __forceinline__ uint64_t pack_f32x2(uint32_t lo, uint32_t hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+// (a.lo * b.lo + c.lo, a.hi * b.hi + c.hi), each a fused multiply-add rounded to nearest even.
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // ---- registers --------------------------------------------------------------
 template <int N>
 __device__ __forceinline__ void reg_alloc() {

@@ -62,11 +62,13 @@ router_logits_kernel(int T, int H, int E, const __nv_bfloat16* __restrict__ x, c
         cp_async_commit();
     };
 
-    float acc[RP_MT][RP_ME];
+    // Accumulators as pairs of tokens (2 i, 2 i + 1) for the packed fp32 FMA: one instruction, two independent
+    // round-to-nearest FMAs, so every sum is bit for bit the one of the scalar form.
+    uint64_t acc2[RP_MT / 2][RP_ME];
 #pragma unroll
-    for (int i = 0; i < RP_MT; ++i)
+    for (int i = 0; i < RP_MT / 2; ++i)
 #pragma unroll
-        for (int j = 0; j < RP_ME; ++j) acc[i][j] = 0.0f;
+        for (int j = 0; j < RP_ME; ++j) acc2[i][j] = 0ull;
 
     const int nkc = H / RP_KC;
     stage(0, 0);
@@ -83,25 +85,34 @@ router_logits_kernel(int T, int H, int E, const __nv_bfloat16* __restrict__ x, c
         const uint8_t* wb = rp_smem + (b * ROWS + ROWS_T + we * RP_ME) * (RP_KC * 2) + lane * 4;
 #pragma unroll
         for (int run = 0; run < RP_KC / 64; ++run) {
-            float xl[RP_MT], xh[RP_MT];
+            uint64_t xl2[RP_MT / 2], xh2[RP_MT / 2];  // elements 2l / 2l+1 of the run for two tokens each
 #pragma unroll
-            for (int i = 0; i < RP_MT; ++i) {
-                const uint32_t u = *reinterpret_cast<const uint32_t*>(xb + i * (RP_KC * 2) + run * 128);
-                xl[i] = __uint_as_float(u << 16);
-                xh[i] = __uint_as_float(u & 0xffff0000u);
+            for (int i = 0; i < RP_MT / 2; ++i) {
+                const uint32_t u0 = *reinterpret_cast<const uint32_t*>(xb + (2 * i) * (RP_KC * 2) + run * 128);
+                const uint32_t u1 = *reinterpret_cast<const uint32_t*>(xb + (2 * i + 1) * (RP_KC * 2) + run * 128);
+                xl2[i] = pack_f32x2(u0 << 16, u1 << 16);
+                xh2[i] = pack_f32x2(u0 & 0xffff0000u, u1 & 0xffff0000u);
             }
 #pragma unroll
             for (int j = 0; j < RP_ME; ++j) {
                 const uint32_t u = *reinterpret_cast<const uint32_t*>(wb + j * (RP_KC * 2) + run * 128);
-                const float wl = __uint_as_float(u << 16), wh = __uint_as_float(u & 0xffff0000u);
+                const uint64_t wl2 = pack_f32x2(u << 16, u << 16), wh2 = pack_f32x2(u & 0xffff0000u, u & 0xffff0000u);
 #pragma unroll
-                for (int i = 0; i < RP_MT; ++i) acc[i][j] = __fmaf_rn(xl[i], wl, acc[i][j]);  // element 2l of the run
+                for (int i = 0; i < RP_MT / 2; ++i) acc2[i][j] = fma_f32x2(xl2[i], wl2, acc2[i][j]);  // element 2l of the run
 #pragma unroll
-                for (int i = 0; i < RP_MT; ++i) acc[i][j] = __fmaf_rn(xh[i], wh, acc[i][j]);  // then element 2l+1
+                for (int i = 0; i < RP_MT / 2; ++i) acc2[i][j] = fma_f32x2(xh2[i], wh2, acc2[i][j]);  // then element 2l+1
             }
         }
         __syncthreads();  // the buffer is refilled two steps from now
     }
+    float acc[RP_MT][RP_ME];
+#pragma unroll
+    for (int i = 0; i < RP_MT / 2; ++i)
+#pragma unroll
+        for (int j = 0; j < RP_ME; ++j) {
+            acc[2 * i][j] = __uint_as_float(static_cast<uint32_t>(acc2[i][j]));
+            acc[2 * i + 1][j] = __uint_as_float(static_cast<uint32_t>(acc2[i][j] >> 32));
+        }
 
     // five pairwise rounds; afterwards every lane holds every logit of the warp tile
 #pragma unroll
