@@ -92,12 +92,17 @@ using GeomFull = Geometry<4, TILE_M, 8, G_EPI_WARPS * G_STORE_WARP_BYTES>;
 // limited by; 512 bytes of output staging per epilogue warp
 using GeomSmall = Geometry<6, 32, 16, G_EPI_WARPS * 512>;
 
-constexpr int F_MAX_TOKENS = GeomSmall::A_ROWS;   // largest batch of fused_small_kernel
+// Row tiles of fused_small_kernel hold at most ST_ROWS = 32 rows (the N of its MMAs); an expert with more rows
+// gets several of them (each streams the expert's weights, the later ones out of L2).  F_MAX_TOKENS is the
+// capacity of the kernel's counters, not the batch size up to which it is the faster path (the host decides).
+constexpr int F_MAX_TOKENS = 256;
+constexpr int F_DEFAULT_MAX_TOKENS = 32;   // up to here the fused kernel is used unless the caller says otherwise
+static_assert(GeomSmall::A_ROWS == ST_ROWS, "the token slot of a stage holds one sub-tile");
 // Largest batch whose routing and permutation run inside fused_small_kernel, by every CTA for itself (one token
 // per warp and round).  Measured against a routing kernel in front: 4-6 us faster per forward up to 13 tokens,
 // equal at 20, 1-6 us slower from 24 tokens up, where a CTA needs two to three rounds.
 constexpr int F_ROUTE_MAX_TOKENS = 16;
-static_assert(F_ROUTE_MAX_TOKENS <= RP_CTA_MAX_TOKENS && F_MAX_TOKENS <= RP_CTA_MAX_TOKENS, "capacity of route_permute_in_cta");
+static_assert(F_ROUTE_MAX_TOKENS <= RP_CTA_MAX_TOKENS, "capacity of route_permute_in_cta");
 static_assert(RP_CTA_SCRATCH_INTS * 4 <= GeomSmall::STAGE_BYTES, "the routing scratch lives in the first pipeline stage");
 
 struct GemmArgs {
@@ -110,6 +115,7 @@ struct GemmArgs {
     const int* num_m_tiles;   // device scalars and tables built by the permute stage
     const int* tile_expert;
     const int* tile_rows;
+    const int* tile_row0;     // fused kernel: first padded row of each (sub-)tile; else null: tile * TILE_M
     const float* a_scale_t;   // [num_kb, row_cap]
     const float* w_scale;     // [E_loc, w_rows/128, num_kb]
     uint8_t* out_fp8;         // GEMM1: [row_cap, I] e4m3
@@ -233,7 +239,8 @@ __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* 
     for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
         const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
         const int wrow = __ldcg(g.tile_expert + m_tile) * g.w_rows_per_expert;
-        const float* a_sc = g.a_scale_t + static_cast<size_t>(m_tile) * TILE_M;
+        const int row0 = FUSED ? __ldcg(g.tile_row0 + m_tile) : m_tile * TILE_M;
+        const float* a_sc = g.a_scale_t + row0;
         // claim the stage of pipeline iteration j: wait until its last reader has finished, announce the bytes
         auto claim = [&](uint32_t j) -> bool {
             const uint32_t s = j % GEO::STAGES, ph = (j / GEO::STAGES) & 1;
@@ -269,7 +276,7 @@ __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* 
             // of the epilogue)
             bulk_load_1d(smem_u32(c.scale_ring + (j % GEO::SCALE_SLOTS) * GEO::A_ROWS),
                          a_sc + static_cast<size_t>(kb) * g.row_cap, GEO::SCALE_BYTES, bar);
-            tma_load_2d(c.smem_base + s * GEO::STAGE_BYTES, tmA, kb * G_BLOCK_K, m_tile * TILE_M, bar);
+            tma_load_2d(c.smem_base + s * GEO::STAGE_BYTES, tmA, kb * G_BLOCK_K, row0, bar);
         };
         int kb = 0;
         if (FUSED && MODE == 2) {
@@ -377,7 +384,7 @@ __device__ __forceinline__ void gather_tiles(const Cta& c, const GemmArgs& g, co
         const int m_tile = tile / g.n_tiles;
         const int rows_valid = __ldcg(g.tile_rows + m_tile);
         // token of row `lane` (scale copy) and source rows of this lane's eight chunks
-        const int my_tok = lane < rows_valid ? __ldcg(f.row_token + static_cast<size_t>(m_tile) * TILE_M + lane) : -1;
+        const int my_tok = lane < rows_valid ? __ldcg(f.row_token + __ldcg(g.tile_row0 + m_tile) + lane) : -1;
         const uint8_t* src_row[GEO::A_ROWS / 4];
 #pragma unroll
         for (int i = 0; i < GEO::A_ROWS / 4; ++i) {
@@ -718,7 +725,8 @@ __device__ __forceinline__ void epilogue_tiles_wm(const Cta& c, const GemmArgs& 
         }
         if (!ok) break;
 
-        const size_t row0 = static_cast<size_t>(m_tile) * TILE_M + th * 16;  // padded row of this thread's token 0
+        const int tile_row0 = __ldcg(g.tile_row0 + m_tile);
+        const size_t row0 = static_cast<size_t>(tile_row0) + th * 16;  // padded row of this thread's token 0
         const int valid = min(16, rows_valid - th * 16);                     // tokens of this thread that exist
         if (MODE == 1) {
             float cc[16];
@@ -823,7 +831,7 @@ __device__ __forceinline__ void epilogue_tiles_wm(const Cta& c, const GemmArgs& 
                 bool last = false;
                 const int r_mine = (warp - 4) + 8 * lane;
                 if (lane < 4 && r_mine < rows_valid) {
-                    tok = __ldcg(f->row_token + static_cast<size_t>(m_tile) * TILE_M + r_mine);
+                    tok = __ldcg(f->row_token + tile_row0 + r_mine);
                     __threadfence();
                     const int before = atomicAdd(f->tok_done + static_cast<size_t>(tok) * g.n_tiles + n, 1);
                     last = before == __ldcg(f->tok_nlocal + tok) - 1;

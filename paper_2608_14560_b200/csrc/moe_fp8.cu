@@ -30,7 +30,7 @@ inline size_t align_up(size_t x, size_t a = WS_ALIGN) { return (x + a - 1) / a *
 
 struct WsLayout {
     size_t topk_idx, topk_w, block_hist, expert_count, expert_offset, padded_offset, tile_expert, tile_rows,
-        num_m_tiles, slot_to_row, row_to_slot, row_token, tok_nlocal, counters, num_counters, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
+        num_m_tiles, slot_to_row, row_to_slot, row_token, tok_nlocal, st_expert, st_row0, st_rows, num_st, counters, num_counters, max_st, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
         stage_scale, stage_logits, stage_out, stage2_hidden, stage2_scale, stage2_logits, stage2_out, total;
     int row_cap, max_m_tiles, max_blocks;
 };
@@ -65,7 +65,14 @@ WsLayout make_layout(const moe_fp8_config& c) {
     L.tok_nlocal = take(Tm * 4);
     // two sets of the fused small-batch kernel's counters (per row tile, per (token, column tile)): a call uses
     // one and zeroes the other for the next call
-    L.num_counters = std::max<size_t>(EL, 1) + static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N);
+    // sub-tiles of at most 32 rows: an expert's padded rows are whole row tiles, four sub-tiles each
+    L.max_st = static_cast<size_t>(L.max_m_tiles) * (TILE_M / ST_ROWS);
+    L.st_expert = take(L.max_st * 4);
+    L.st_row0 = take(L.max_st * 4);
+    L.st_rows = take(L.max_st * 4);
+    L.num_st = take(4);
+    // (a batch the fused kernel takes has at most EL + F_MAX_TOKENS * 8 / 32 sub-tiles)
+    L.num_counters = std::min<size_t>(L.max_st, EL + F_MAX_TOKENS / 4) + static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N);
     L.counters = take(2 * L.num_counters * 4);
     L.status = take(8);  // device status word, then the ticket counter of route_permute_kernel
     L.a1 = take(rc * H);
@@ -108,7 +115,7 @@ struct moe_fp8_handle_s {
     int fault_skip_it;         // test hook, see moe_fp8_debug_set_fault
     long long fault_wait_limit;
     cudaEvent_t ev[NUM_STAGES_MAX + 1];
-    bool small_fusion;
+    int fused_max_tokens;   // batches of at most this many tokens take the fused kernel (0: never)
     unsigned long long fused_calls;
     // moe_fp8_forward_host_async: copy streams and the events that order the two staging sets
     bool pipe_ready;
@@ -174,6 +181,10 @@ PermuteMeta meta_of(moe_fp8_handle_t h) {
     m.row_to_slot = at<int>(h, h->L.row_to_slot);
     m.row_token = at<int>(h, h->L.row_token);
     m.tok_nlocal = at<int>(h, h->L.tok_nlocal);
+    m.st_expert = at<int>(h, h->L.st_expert);
+    m.st_row0 = at<int>(h, h->L.st_row0);
+    m.st_rows = at<int>(h, h->L.st_rows);
+    m.num_st = at<int>(h, h->L.num_st);
     return m;
 }
 
@@ -273,7 +284,7 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     h->cfg = *cfg;
     h->L = make_layout(*cfg);
     h->sm_count = sms;
-    h->small_fusion = true;
+    h->fused_max_tokens = F_DEFAULT_MAX_TOKENS;
     h->fused_calls = 0;
     h->fault_skip_it = -1;
     h->fault_wait_limit = WAIT_LIMIT_CLOCKS;
@@ -398,7 +409,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     mark();
     // Batches of at most F_MAX_TOKENS tokens: gather, both GEMMs and the combine in one kernel; up to
     // F_ROUTE_MAX_TOKENS that kernel also routes and permutes (every CTA for itself: one launch per forward).
-    const bool fused = h->small_fusion && T <= F_MAX_TOKENS;
+    const bool fused = T <= h->fused_max_tokens;
     const bool route_in_fused = fused && T <= F_ROUTE_MAX_TOKENS;
     int *counters = nullptr, *counters_next = nullptr;
     if (fused) {
@@ -489,7 +500,12 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         f.topk_w = topk_w;
         f.tok_nlocal = m.tok_nlocal;
         f.ready = counters;
-        f.tok_done = counters + std::max(EL, 1);
+        f.tok_done = counters + (h->L.num_counters - static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N));
+        // the fused kernel works on sub-tiles of at most 32 rows
+        g1.num_m_tiles = g2.num_m_tiles = m.num_st;
+        g1.tile_expert = g2.tile_expert = m.st_expert;
+        g1.tile_rows = g2.tile_rows = m.st_rows;
+        g1.tile_row0 = g2.tile_row0 = m.st_row0;
         f.out = static_cast<__nv_bfloat16*>(out);
         f.route = route_in_fused;
         f.E_loc = EL;
@@ -552,7 +568,8 @@ int moe_fp8_debug_set_fault(moe_fp8_handle_t h, int skip_iteration, long long wa
 
 int moe_fp8_set_small_batch_fusion(moe_fp8_handle_t h, int enable) {
     if (!h) return MOE_FP8_ERR_BAD_ARG;
-    h->small_fusion = enable != 0;
+    if (enable < 0 || enable > F_MAX_TOKENS) return MOE_FP8_ERR_BAD_ARG;
+    h->fused_max_tokens = enable == 0 ? 0 : enable == 1 ? F_DEFAULT_MAX_TOKENS : enable;
     return MOE_FP8_OK;
 }
 

@@ -30,7 +30,13 @@ struct PermuteMeta {
     int* row_to_slot;    // [T*8] canonical row -> slot id (first S entries valid)
     int* row_token;      // [row_cap] padded row -> token (valid rows only)
     int* tok_nlocal;     // [T] local slots of each token (small batches only: route_permute_kernel / _in_cta)
+    // small batches only, for the fused kernel: the row tiles cut into sub-tiles of at most 32 rows
+    int* st_expert;      // [max sub-tiles] local expert
+    int* st_row0;        // [max sub-tiles] first padded row (a multiple of 32)
+    int* st_rows;        // [max sub-tiles] valid rows (1..32)
+    int* num_st;         // [1]
 };
+constexpr int ST_ROWS = 32;
 
 // Bit t of mask[e] says: token t of this block routes to local expert e.  The
 // popcount below a token's bit is its stable rank inside the block.
@@ -169,6 +175,7 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
     extern __shared__ uint32_t dyn_smem[];
     __shared__ int s_cnt[P_MAX_LOCAL + 1];
     __shared__ int s_pad[P_MAX_LOCAL + 1];
+    __shared__ int s_st[P_MAX_LOCAL + 1];
     __shared__ int s_last;
     const int tid = threadIdx.x, lane = tid & 31;
     if (blockIdx.x == 0 && tid == 0) *status = DEV_OK;  // first kernel of a forward: clear the fault word
@@ -234,17 +241,20 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
     }
     __syncthreads();
     if (tid == 0) {  // 256 entries: a serial scan is a few hundred cycles
-        int a = 0, p = 0;
+        int a = 0, p = 0, st = 0;
         for (int i = 0; i < E_loc; ++i) {
             const int c = s_cnt[i], q = s_pad[i];
             s_cnt[i] = a;
             s_pad[i] = p;
+            s_st[i] = st;
             a += c;
             p += q;
+            st += (c + ST_ROWS - 1) / ST_ROWS;
         }
         s_cnt[E_loc] = a;
         s_pad[E_loc] = p;
         *m.num_m_tiles = p / TILE_M;
+        *m.num_st = st;
         m.expert_offset[E_loc] = a;
         m.padded_offset[E_loc] = p;
     }
@@ -257,6 +267,11 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
         for (int i = 0; i * TILE_M < total; ++i) {
             m.tile_expert[t0 + i] = e;
             m.tile_rows[t0 + i] = min(TILE_M, total - i * TILE_M);
+        }
+        for (int i = 0; i * ST_ROWS < total; ++i) {
+            m.st_expert[s_st[e] + i] = e;
+            m.st_row0[s_st[e] + i] = s_pad[e] + i * ST_ROWS;
+            m.st_rows[s_st[e] + i] = min(ST_ROWS, total - i * ST_ROWS);
         }
     }
     for (int t = tid; t < T; t += blockDim.x) {
@@ -287,6 +302,7 @@ __global__ void __launch_bounds__(P_TAIL_THREADS) route_permute_kernel(
     }
 }
 static_assert(P_TAIL_THREADS == P_MAX_LOCAL, "the tail keeps one expert's count per thread");
+static_assert(TILE_M % ST_ROWS == 0, "sub-tiles do not straddle row tiles");
 
 // Stages 1 and 2 for a batch of at most 32 tokens, computed by ONE thread block for itself: every CTA of the
 // fused small-batch kernel runs this on the same inputs and writes the same tables (to the same addresses, with
@@ -372,14 +388,19 @@ __device__ __forceinline__ void route_permute_in_cta(int* scratch, int T, int E_
         m.expert_count[tid] = total;
         m.expert_offset[tid] = s_cnt[tid];
         m.padded_offset[tid] = s_pad[tid];
+        // at most RP_CTA_MAX_TOKENS = 32 rows per expert: one row tile, which is also its only sub-tile
         const int t0 = s_pad[tid] / TILE_M;
-        for (int i = 0; i * TILE_M < total; ++i) {
-            m.tile_expert[t0 + i] = tid;
-            m.tile_rows[t0 + i] = min(TILE_M, total - i * TILE_M);
+        if (total > 0) {
+            m.tile_expert[t0] = tid;
+            m.tile_rows[t0] = total;
+            m.st_expert[t0] = tid;
+            m.st_row0[t0] = s_pad[tid];
+            m.st_rows[t0] = total;
         }
     }
     if (tid == 0) {  // entries past E_loc count nothing, so entry E_loc already holds the totals
         *m.num_m_tiles = s_pad[E_loc] / TILE_M;
+        *m.num_st = s_pad[E_loc] / TILE_M;
         m.expert_offset[E_loc] = s_cnt[E_loc];
         m.padded_offset[E_loc] = s_pad[E_loc];
     }
