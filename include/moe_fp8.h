@@ -174,15 +174,20 @@ int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w
                          int* status_word, void* stream);
 
 /*
- * Batches of at most 32 tokens run the gather of stage 2, both GEMMs of stage 3 and the combine of stage 4 as
- * ONE kernel (the paper's short regime, T = 1-16, is bounded by routing and launch overhead, and it names
- * fusing the scatter into GEMM2's epilogue as the next step; in that kernel the CTA that stores the last local
- * row of a token sums the token's rows in routing order, so results stay bit-identical to the separate
- * kernels).  Up to 16 tokens that kernel also does stages 1 and 2 -- every CTA routes and permutes the whole
- * batch for itself and all write the same tables -- so a forward is a single launch; from 17 to 32 tokens a
- * routing kernel runs in front of it.  The kernel's cross-CTA counters live in the workspace in two sets: a call
- * uses one and zeroes the other, so a call that gave up on a bounded wait does not disturb later ones.
- * On by default; enable = 0 makes such batches take the separate kernels too.
+ * Small batches run the gather of stage 2, both GEMMs of stage 3 and the combine of stage 4 as ONE kernel (the
+ * paper's short regime, T = 1-16, is bounded by routing and launch overhead, and it names fusing the scatter
+ * into GEMM2's epilogue as the next step; in that kernel the CTA that stores the last local row of a token
+ * sums the token's rows in routing order, so results stay bit-identical to the separate kernels).  Its MMAs
+ * take the weights on the M side and a tile's at most 32 token rows on the N side; an expert with more rows is
+ * worked on as several such tiles.  Up to 16 tokens that kernel also does stages 1 and 2 -- every CTA routes
+ * and permutes the whole batch for itself and all write the same tables -- so a forward is a single launch;
+ * above that a routing kernel runs in front of it.  The kernel's cross-CTA counters live in the workspace in two
+ * sets: a call uses one and zeroes the other, so a call that gave up on a bounded wait does not disturb later
+ * ones.
+ * enable = 1 (the default): batches of at most 80 tokens take the fused kernel (measured faster up to there
+ * for uniform and for skewed routing; with well balanced routing it stays faster up to about 200 tokens);
+ * enable = 0: every batch takes the separate kernels; enable = 2..256: batches of at most that many tokens
+ * take the fused kernel.  Other values: MOE_FP8_ERR_BAD_ARG.
  */
 int moe_fp8_set_small_batch_fusion(moe_fp8_handle_t h, int enable);
 

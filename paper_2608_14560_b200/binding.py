@@ -227,9 +227,10 @@ class MoeFp8:
             self._stream(stream)))
         return host_out
 
-    def set_small_batch_fusion(self, enable: bool):
-        """moe_fp8_set_small_batch_fusion: batches of <= 32 tokens as one fused kernel (default; a single launch per forward
-        up to 16 tokens) or as separate ones."""
+    def set_small_batch_fusion(self, enable):
+        """moe_fp8_set_small_batch_fusion: False / 0 = separate kernels at every batch size; True / 1 = the fused
+        kernel up to the default limit (80 tokens; a single launch per forward up to 16 tokens); 2..256 = the
+        fused kernel up to that many tokens."""
         self._check(self.lib.moe_fp8_set_small_batch_fusion(self.handle, int(enable)))
 
     def debug_set_fault(self, skip_iteration: int = -1, wait_clocks: int = 0):

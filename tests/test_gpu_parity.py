@@ -324,10 +324,11 @@ def test_from_hidden_benchmark_shapes(cuda_device, cfg, n_sample):
     assert S > 0
 
 
-# ---- batches of at most 32 tokens: gather, both GEMMs and the combine as one kernel; up to 16 tokens that ----
+# ---- batches of at most 80 tokens: gather, both GEMMs and the combine as one kernel; up to 16 tokens that ----
 # ---- kernel also routes and permutes (every CTA for itself), and the forward is a single launch -------------
 @pytest.mark.parametrize("tokens,kw", [(1, {}), (5, {}), (12, {}), (13, {}), (16, {"local_expert_offset": 64}),
-                                       (17, {}), (32, {}), (23, {"skew": True})])
+                                       (17, {}), (32, {}), (23, {"skew": True}), (33, {}), (64, {"skew": True}),
+                                       (80, {}), (80, {"skew": True, "local_expert_offset": 32})])
 def test_fused_small_batch_kernel_is_bit_identical_to_the_separate_kernels(cuda_device, tokens, kw):
     wl = _wl(tokens, seed=80 + tokens, **kw)
     inp = syn.make_inputs(wl, cuda_device)
@@ -350,7 +351,7 @@ def test_fused_small_batch_kernel_transposed_scales_and_full_size_layer(cuda_dev
     inp = syn.make_inputs(wl, cuda_device)
     run_and_compare(wl, cuda_device, inp=dict(inp, hidden_scale=inp["hidden_scale"].t().contiguous()), hidden_scale_layout=1)
     base = syn.CONFIGS[0]
-    for tokens in (1, 16, 32):
+    for tokens in (1, 16, 32, 64):
         wl = syn.Workload(f"dsv3_T{tokens}_E32", tokens, base.dims, base.seed + tokens)
         inp = syn.make_inputs(wl, cuda_device)
         eng = make_engine(wl, cuda_device)
@@ -364,6 +365,24 @@ def test_fused_small_batch_kernel_transposed_scales_and_full_size_layer(cuda_dev
         assert torch.equal(got.view(torch.int16), want.view(torch.int16))
         run_and_compare(wl, cuda_device, inp=inp, eng=eng)
         eng.close()
+
+
+@pytest.mark.parametrize("tokens,kw", [(200, {"skew": True}), (256, {}), (130, {"skew": True, "local_expert_offset": 96})])
+def test_fused_kernel_with_a_raised_limit_cuts_experts_into_sub_tiles(cuda_device, tokens, kw):
+    # beyond the default limit the caller may still ask for the fused kernel (up to 256 tokens): experts with
+    # more than 32 rows are then worked on as several sub-tiles of 32 rows
+    wl = _wl(tokens, seed=170 + tokens, **kw)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device)
+    want = eng.forward(inp).clone()
+    assert eng.last_launch_count() == 5
+    eng.set_small_batch_fusion(256)
+    got = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert eng.status() == 0 and eng.last_launch_count() == 2
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    dbg = run_and_compare(wl, cuda_device, inp=inp, eng=eng)
+    eng.close()
 
 
 def test_a_wait_that_runs_out_in_the_fused_small_batch_kernel(cuda_device):
@@ -391,7 +410,7 @@ def test_a_wait_that_runs_out_in_the_fused_small_batch_kernel(cuda_device):
 def test_small_batches_of_changing_size_share_the_alternating_counters(cuda_device):
     # one handle, batch sizes on both sides of every launch scheme (one launch, routing kernel + fused kernel,
     # separate kernels) in turn: what one forward leaves in the workspace must not reach the next
-    sizes = [7, 30, 3, 40, 16, 17, 1, 32, 12, 33, 9]
+    sizes = [7, 30, 3, 90, 16, 17, 1, 80, 12, 81, 9, 40]
     base = _wl(max(sizes), seed=47)
     inp = syn.make_inputs(base, cuda_device)
     eng = make_engine(base, cuda_device)
@@ -404,7 +423,7 @@ def test_small_batches_of_changing_size_share_the_alternating_counters(cuda_devi
         want = ref.forward(part).clone()
         torch.cuda.synchronize()
         assert eng.status() == 0 and ref.status() == 0
-        assert eng.last_launch_count() == (1 if t <= 16 else 2 if t <= 32 else 5), t
+        assert eng.last_launch_count() == (1 if t <= 16 else 2 if t <= 80 else 5), t
         assert torch.equal(got.view(torch.int16), want.view(torch.int16)), t
     eng.close()
     ref.close()
