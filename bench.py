@@ -40,10 +40,11 @@ FP8_DATASHEET_TFLOPS = 4500.0
 HBM_DATASHEET_GBS = 8000.0
 # Measured DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch divided by the algorithmic
 # bytes of the same launch, from the committed ncu captures (see profiles/): the weight-streaming regime was
-# captured on the T = 64 workload itself, the tensor-bound regime on a reduced case (32 local experts) whose
-# traffic is scaled to a full launch by the algorithmic bytes, since both grow with the experts and rows.
+# captured on the T = 8 and T = 64 workloads (fused kernel) and on the T = 1024 workload (the two GEMM kernels)
+# themselves, the tensor-bound regime on a reduced case (32 local experts) whose traffic is scaled to a full
+# launch by the algorithmic bytes, since both grow with the experts and rows.
 NCU_TRAFFIC_RATIO = {
-    ("hbm", "gemm1_swiglu_quant"): 1.035, ("hbm", "gemm2"): 1.02,
+    ("hbm", "gemm1_swiglu_quant"): 1.04, ("hbm", "gemm2"): 1.02,
     ("tensor", "gemm1_swiglu_quant"): 1.31, ("tensor", "gemm2"): 0.99,
     ("hbm", "fused_small"): 1.00,
 }
