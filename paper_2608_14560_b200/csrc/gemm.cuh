@@ -25,7 +25,7 @@
 //
 // Two kernels are built from these roles:
 //   grouped_gemm_kernel<MODE>   one GEMM per launch (any batch size);
-//   fused_small_kernel          batches of at most F_MAX_TOKENS tokens: the gather of stage 2, GEMM1, GEMM2
+//   fused_small_kernel          small batches (the host decides up to which size): the gather of stage 2, GEMM1, GEMM2
 //               and the weighted combine of stage 4 in ONE launch, with the operands swapped (weights on the
 //               M side of the MMA, the tile's at most 32 token rows on the N side; see "weights on M" below).
 //               Every CTA first works through its GEMM1 tiles, then its GEMM2 tiles.  Warp 3 gathers the (few)
@@ -940,9 +940,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
 }
 
-// Gather + GEMM1 + GEMM2 + combine in one launch for batches of at most F_MAX_TOKENS tokens (see the head of
-// this file).  tmA2 / tmOut describe GEMM1's output buffer for loads (32-row boxes) / stores, tmB1 / tmB2 the
-// two weight tensors.
+// Gather + GEMM1 + GEMM2 + combine in one launch for small batches, at most F_MAX_TOKENS tokens (see the head of
+// this file).  tmA2 describes GEMM1's output buffer for loads (32-row boxes), tmB1 / tmB2 the two weight
+// tensors.
 __global__ void __launch_bounds__(G_THREADS, 1)
 fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmB1,
                    const __grid_constant__ CUtensorMap tmB2, const GemmArgs g1, const GemmArgs g2, const FusedArgs f) {

@@ -121,7 +121,7 @@ struct moe_fp8_handle_s {
     bool pipe_ready;
     unsigned pipe_calls;
     cudaStream_t s_in, s_out;
-    cudaEvent_t ev_in[2], ev_compute[2], ev_out[2];         // batches of at most F_MAX_TOKENS tokens take the single fused kernel
+    cudaEvent_t ev_in[2], ev_compute[2], ev_out[2];
 };
 
 namespace {
@@ -407,7 +407,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     } while (0)
     h->stage_times_valid = false;
     mark();
-    // Batches of at most F_MAX_TOKENS tokens: gather, both GEMMs and the combine in one kernel; up to
+    // Batches of at most fused_max_tokens tokens: gather, both GEMMs and the combine in one kernel; up to
     // F_ROUTE_MAX_TOKENS that kernel also routes and permutes (every CTA for itself: one launch per forward).
     const bool fused = T <= h->fused_max_tokens;
     const bool route_in_fused = fused && T <= F_ROUTE_MAX_TOKENS;
