@@ -385,13 +385,14 @@ def test_fused_kernel_with_a_raised_limit_cuts_experts_into_sub_tiles(cuda_devic
     eng.close()
 
 
-def test_a_wait_that_runs_out_in_the_fused_small_batch_kernel(cuda_device):
-    wl = _wl(16, seed=43)
+@pytest.mark.parametrize("tokens,launches", [(16, 1), (48, 2)])
+def test_a_wait_that_runs_out_in_the_fused_small_batch_kernel(cuda_device, tokens, launches):
+    wl = _wl(tokens, seed=43)
     inp = syn.make_inputs(wl, cuda_device)
     eng = make_engine(wl, cuda_device)
     want = eng.forward(inp).clone()
     torch.cuda.synchronize()
-    assert eng.status() == 0 and eng.last_launch_count() == 1
+    assert eng.status() == 0 and eng.last_launch_count() == launches
     eng.debug_set_fault(skip_iteration=1, wait_clocks=1 << 20)
     eng.forward(inp)
     torch.cuda.synchronize()
