@@ -70,10 +70,10 @@ int moe_fp8_destroy(moe_fp8_handle_t h);
 /* Bytes of device scratch needed for cfg.max_tokens tokens. */
 size_t moe_fp8_workspace_bytes(moe_fp8_handle_t h);
 /* Hands the library a caller-owned device buffer (1024-byte aligned) that must
- * stay valid until it is replaced or the handle destroyed.  The call zeroes two
- * control words in it and waits for the device (cudaDeviceSynchronize); after that the
- * contents belong to the library: a counter lives there between forwards, so
- * the caller must not write into the buffer. */
+ * stay valid until it is replaced or the handle destroyed.  The call zeroes the
+ * control words and counters in it and waits for the device (cudaDeviceSynchronize);
+ * after that the contents belong to the library: counters live there between
+ * forwards, so the caller must not write into the buffer. */
 int moe_fp8_set_workspace(moe_fp8_handle_t h, void* dev_workspace, size_t bytes);
 
 /*
@@ -93,6 +93,10 @@ int moe_fp8_set_workspace(moe_fp8_handle_t h, void* dev_workspace, size_t bytes)
  *                        weights were normalised over all 8 selected experts
  *   scaling_factor routed scaling factor (2.5)
  *   out            bf16 [T, H], fully overwritten (zeros for tokens without a local expert)
+ *
+ * All pointers are device pointers, 16-byte aligned; nothing is copied or kept beyond the call's kernels.
+ * Forwards on one handle share its workspace: their kernels must not overlap on the GPU (one stream, or
+ * streams ordered with events); use one handle per concurrent stream otherwise.
  */
 int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const float* hidden_scale,
                     const float* router_logits, const void* routing_bias, const void* w13,
