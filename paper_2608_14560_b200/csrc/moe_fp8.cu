@@ -414,7 +414,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
     int *counters = nullptr, *counters_next = nullptr;
     if (fused) {
         // this call's counter set is zero: the fused call before it zeroed it (set_workspace for the first two)
-        const size_t set = h->fused_calls++ & 1;
+        const size_t set = h->fused_calls & 1;  // (advanced once the fused kernel is enqueued)
         counters = at<int>(h, h->L.counters) + set * h->L.num_counters;
         counters_next = at<int>(h, h->L.counters) + (set ^ 1) * h->L.num_counters;
     }
@@ -525,6 +525,7 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         mark();  // combine
         MOE_LAUNCH(fused_small_kernel, h->sm_count, G_THREADS, GeomSmall::SMEM_BYTES, stream, pdl, h->tm_a2_small,
                    h->tm_w13, h->tm_w2, g1, g2, f);
+        ++h->fused_calls;  // only a kernel that runs zeroes the other counter set
         mark();
     } else {
         {  // stage 2, continued: gather
