@@ -47,6 +47,26 @@ def test_local_expert_offsets(cuda_device, off, eloc):
     run_and_compare(_wl(200, dims, seed=off + eloc, local_expert_offset=off), cuda_device)
 
 
+@pytest.mark.parametrize("tokens,eloc,off", [(9, 256, 0), (60, 256, 0), (80, 3, 5), (33, 1, 0), (70, 1, 7)])
+def test_fused_small_batch_kernel_with_many_and_with_few_local_experts(cuda_device, tokens, eloc, off):
+    # all experts local: a couple of hundred one- or two-row tiles; one local expert: every local row in one
+    # expert, i.e. up to three sub-tiles of the same weights
+    dims = dataclasses.replace(SMALL, num_local_experts=eloc)
+    wl = _wl(tokens, dims, seed=300 + tokens + eloc, local_expert_offset=off)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device)
+    got = eng.forward(inp).clone()
+    assert eng.last_launch_count() <= 2
+    eng.set_small_batch_fusion(False)
+    want = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert eng.status() == 0 and eng.last_launch_count() == 5
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    eng.set_small_batch_fusion(True)
+    run_and_compare(wl, cuda_device, inp=inp, eng=eng)
+    eng.close()
+
+
 def test_scale_layout_and_gate_order_flags(cuda_device):
     wl = _wl(97, seed=3)
     inp = syn.make_inputs(wl, cuda_device)
