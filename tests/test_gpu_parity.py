@@ -467,18 +467,19 @@ def test_every_token_count_of_the_bench_sweep(cuda_device):
     eng.close()
 
 
-def test_pipelined_host_entry_point_matches_device_entry_point(cuda_device):
+@pytest.mark.parametrize("tokens", [300, 40, 9])  # separate kernels | fused behind the routing kernel | one launch
+def test_pipelined_host_entry_point_matches_device_entry_point(cuda_device, tokens):
     # five steps through moe_fp8_forward_host_async with three different batches in rotation (two staging sets
     # alternate inside the library): every step's host result equals the device-buffer forward of its batch
-    wl = _wl(300, seed=13)
-    batches = [syn.make_inputs(_wl(300, seed=13 + i), cuda_device) for i in range(3)]
+    wl = _wl(tokens, seed=13)
+    batches = [syn.make_inputs(_wl(tokens, seed=13 + i), cuda_device) for i in range(3)]
     weights = batches[0]
     eng = make_engine(wl, cuda_device)
     want = []
     for b in batches:
         want.append(eng.forward({**weights, **{k: b[k] for k in ("hidden_fp8", "hidden_scale", "router_logits")}}).cpu())
     host_acts = [{k: b[k].cpu().pin_memory() for k in ("hidden_fp8", "hidden_scale", "router_logits")} for b in batches]
-    host_outs = [torch.empty(300, 512, dtype=torch.bfloat16).pin_memory() for _ in range(5)]
+    host_outs = [torch.empty(tokens, 512, dtype=torch.bfloat16).pin_memory() for _ in range(5)]
     for i in range(5):
         eng.forward_host_async(host_acts[i % 3], weights, host_outs[i])
     eng.host_sync()
