@@ -196,6 +196,14 @@ int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w
 int moe_fp8_set_small_batch_fusion(moe_fp8_handle_t h, int enable);
 
 /*
+ * Inside the two large-tile GEMM kernels a row tile that holds at most 32 rows (an expert's short last tile) is
+ * worked on with the operands swapped -- weights on the M side of the MMAs, the 32 token rows on N, a 64-column
+ * accumulator -- instead of as a full 128-row tile: same arithmetic, bit-identical results, less tensor and
+ * epilogue time.  This hook sets the batch size from which that applies (min_tokens = 0: never).
+ */
+int moe_fp8_debug_set_short_tiles(moe_fp8_handle_t h, int min_tokens);
+
+/*
  * Test hook for the failure path of the bounded device waits (every wait on an mbarrier inside the GEMM
  * kernels gives up after a limit, records a fault code in the status word and lets the kernel return with
  * its tensor memory released).  skip_iteration >= 0: in the next forwards the copy producer of every CTA

@@ -96,6 +96,8 @@ using GeomSmall = Geometry<6, 32, 16, G_EPI_WARPS * 512>;
 // gets several of them (each streams the expert's weights, the later ones out of L2).  F_MAX_TOKENS is the
 // capacity of the kernel's counters, not the batch size up to which it is the faster path (the host decides).
 constexpr int F_MAX_TOKENS = 256;
+// From this batch size up the large-tile GEMM kernels run row tiles of at most 32 rows with the weights on M.
+constexpr int SHORT_TILE_MIN_TOKENS = 1;
 // Up to here the fused kernel is used unless the caller says otherwise.  Measured against the separate kernels
 // (cold step): 9-17 % faster from 34 to 80 tokens with uniform routing, 13-16 % faster at 40-64 tokens with
 // skewed routing, 3-6 % slower at exactly 33 and at 80 skewed tokens (hot experts need a second or third
@@ -109,6 +111,9 @@ constexpr int F_ROUTE_MAX_TOKENS = 16;
 static_assert(F_ROUTE_MAX_TOKENS <= RP_CTA_MAX_TOKENS, "capacity of route_permute_in_cta");
 static_assert(RP_CTA_SCRATCH_INTS * 4 <= GeomSmall::STAGE_BYTES, "the routing scratch lives in the first pipeline stage");
 
+constexpr int WM_TOKENS = 32;                       // weights-on-M tiles: N of the MMA, token rows of a tile
+constexpr int WM_BUF_COLS = 2 * WM_TOKENS;          // their TMEM columns per K-block: two weight-row blocks
+
 struct GemmArgs {
     int num_kb;               // K / 128
     int n_tiles;              // output tiles along N per row tile
@@ -120,6 +125,8 @@ struct GemmArgs {
     const int* tile_expert;
     const int* tile_rows;
     const int* tile_row0;     // fused kernel: first padded row of each (sub-)tile; else null: tile * TILE_M
+    int wm_rows;              // large-tile kernel: row tiles with at most this many rows (0 or 32) run with the
+                              // weights on the M side of the MMAs, see epilogue_tile_wm
     const float* a_scale_t;   // [num_kb, row_cap]
     const float* w_scale;     // [E_loc, w_rows/128, num_kb]
     uint8_t* out_fp8;         // GEMM1: [row_cap, I] e4m3
@@ -237,14 +244,18 @@ __device__ __forceinline__ void gemm_cta_setup(Cta& c, uint8_t* smem_raw, int fu
 template <int MODE, bool FUSED, class GEO>
 __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* tmA, const CUtensorMap* tmB,
                                                const GemmArgs& g, const FusedArgs* f, int ready_target, TileRange tr,
-                                               uint32_t& it, bool& ok) {
+                                               uint32_t& it, bool& ok, const CUtensorMap* tmA_short = nullptr) {
     GemmCtrl* ctrl = c.ctrl;
-    constexpr uint32_t TX_BYTES = (FUSED && MODE == 1) ? G_B_BYTES : GEO::STAGE_BYTES + GEO::SCALE_BYTES;
     for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
         const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
         const int wrow = __ldcg(g.tile_expert + m_tile) * g.w_rows_per_expert;
         const int row0 = FUSED ? __ldcg(g.tile_row0 + m_tile) : m_tile * TILE_M;
         const float* a_sc = g.a_scale_t + row0;
+        // a short row tile of the large-tile kernel: 32 token rows fetched, weights laid out for the M side
+        const bool wm = !FUSED && g.wm_rows > 0 && __ldcg(g.tile_rows + m_tile) <= g.wm_rows;
+        const uint32_t TX_BYTES = (FUSED && MODE == 1) ? G_B_BYTES
+                                  : wm ? WM_TOKENS * G_BLOCK_K + WM_TOKENS * 4 + G_B_BYTES
+                                       : GEO::STAGE_BYTES + GEO::SCALE_BYTES;
         // claim the stage of pipeline iteration j: wait until its last reader has finished, announce the bytes
         auto claim = [&](uint32_t j) -> bool {
             const uint32_t s = j % GEO::STAGES, ph = (j / GEO::STAGES) & 1;
@@ -265,8 +276,8 @@ __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* 
                 // weights on N: gate[0,64) | up[0,64) | gate[64,128) | up[64,128); on M (fused kernel):
                 // gate[0,128) | up[0,128)
                 tma_load_2d(b_dst, tmB, k0, gr, bar);
-                tma_load_2d(b_dst + G_B_BYTES / 4, tmB, k0, FUSED ? gr + 64 : ur, bar);
-                tma_load_2d(b_dst + G_B_BYTES / 2, tmB, k0, FUSED ? ur : gr + 64, bar);
+                tma_load_2d(b_dst + G_B_BYTES / 4, tmB, k0, (FUSED || wm) ? gr + 64 : ur, bar);
+                tma_load_2d(b_dst + G_B_BYTES / 2, tmB, k0, (FUSED || wm) ? ur : gr + 64, bar);
                 tma_load_2d(b_dst + 3 * G_B_BYTES / 4, tmB, k0, ur + 64, bar);
             } else {
                 const int br = wrow + n * G_TILE_N;
@@ -279,8 +290,8 @@ __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* 
             // (the scale slot is free: the ring exceeds the stages + accumulators the producer can be ahead
             // of the epilogue)
             bulk_load_1d(smem_u32(c.scale_ring + (j % GEO::SCALE_SLOTS) * GEO::A_ROWS),
-                         a_sc + static_cast<size_t>(kb) * g.row_cap, GEO::SCALE_BYTES, bar);
-            tma_load_2d(c.smem_base + s * GEO::STAGE_BYTES, tmA, kb * G_BLOCK_K, row0, bar);
+                         a_sc + static_cast<size_t>(kb) * g.row_cap, wm ? WM_TOKENS * 4 : GEO::SCALE_BYTES, bar);
+            tma_load_2d(c.smem_base + s * GEO::STAGE_BYTES, wm ? tmA_short : tmA, kb * G_BLOCK_K, row0, bar);
         };
         int kb = 0;
         if (FUSED && MODE == 2) {
@@ -332,8 +343,11 @@ template <class GEO>
 __device__ __forceinline__ void issuer_tiles(const Cta& c, const GemmArgs& g, TileRange tr, uint32_t mine,
                                              uint32_t& it, bool& ok) {
     GemmCtrl* ctrl = c.ctrl;
-    const uint32_t idesc = umma_idesc_f8(TILE_M, G_TILE_N);
+    const uint32_t idesc = umma_idesc_f8(TILE_M, G_TILE_N), idesc_wm = umma_idesc_f8(TILE_M, WM_TOKENS);
     for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        // a short row tile: the stage's weight rows are the M side (two blocks of 128), its 32 token rows the N
+        // side; the accumulator is the first 64 columns of the buffer
+        const bool wm = g.wm_rows > 0 && __ldcg(g.tile_rows + tile / g.n_tiles) <= g.wm_rows;
         for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
             if ((it & 1) != mine) continue;
             const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
@@ -355,9 +369,18 @@ __device__ __forceinline__ void issuer_tiles(const Cta& c, const GemmArgs& g, Ti
                 break;
             }
             tc_fence_after();
+            if (wm) {
+                const uint64_t w1_desc = umma_desc_sw128(a_addr + GEO::A_BYTES + G_B_BYTES / 2);
 #pragma unroll
-            for (int k = 0; k < G_BLOCK_K / 32; ++k)  // 32 K-bytes per instruction: +2 in 16-B units
-                umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k > 0);
+                for (int k = 0; k < G_BLOCK_K / 32; ++k) umma_f8(d_tmem, b_desc + 2 * k, a_desc + 2 * k, idesc_wm, k > 0);
+#pragma unroll
+                for (int k = 0; k < G_BLOCK_K / 32; ++k)
+                    umma_f8(d_tmem + WM_TOKENS, w1_desc + 2 * k, a_desc + 2 * k, idesc_wm, k > 0);
+            } else {
+#pragma unroll
+                for (int k = 0; k < G_BLOCK_K / 32; ++k)  // 32 K-bytes per instruction: +2 in 16-B units
+                    umma_f8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k > 0);
+            }
             umma_commit(smem_u32(&ctrl->done[s]));
         }
     }
@@ -449,6 +472,10 @@ __device__ __forceinline__ bool epilogue_rendezvous(const Cta& c, uint32_t& n) {
     return ok;
 }
 
+template <int MODE, bool FUSED, class GEO, bool SHARED>
+__device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, int m_tile, int n,
+                                                 uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter);
+
 // ---------------- epilogue warps ----------------
 // MODE 1: gate/up projection + SwiGLU + re-quantisation; tmOut describes the e4m3 output [row_cap, I] for
 //         64-byte x 32-row TMA stores.
@@ -473,6 +500,11 @@ __device__ __forceinline__ void epilogue_tiles(const Cta& c, const CUtensorMap* 
         const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
         const int e = __ldcg(g.tile_expert + m_tile);
         const int rows_valid = __ldcg(g.tile_rows + m_tile);
+        if (g.wm_rows > 0 && rows_valid <= g.wm_rows) {  // a short row tile, worked on with the weights on M
+            uint32_t unused = 0;
+            ok = epilogue_tile_wm<MODE, false, GEO, true>(c, g, nullptr, m_tile, n, it, tile_iter, unused);
+            continue;
+        }
         const size_t row = static_cast<size_t>(m_tile) * TILE_M + r_in_tile;
         const int sblocks = g.w_rows_per_expert / 128;
         // weight-scale rows of this thread's first / second 64 columns
@@ -615,8 +647,6 @@ __device__ __forceinline__ void epilogue_tiles(const Cta& c, const CUtensorMap* 
 // so the hand-over latencies overlap six deep, and every epilogue thread owns one weight row (an output
 // column) for 16 tokens -- 32 loads and 32 FMAs per K-block instead of 128, evenly over all eight warps.
 // Element for element the arithmetic is the one of the other orientation.
-constexpr int WM_TOKENS = 32;                       // N of the MMA: token rows of a tile
-constexpr int WM_BUF_COLS = 2 * WM_TOKENS;          // TMEM columns per K-block: two weight-row blocks
 static_assert(G_MAX_STAGES * WM_BUF_COLS <= static_cast<int>(G_TMEM_COLS), "one accumulator buffer per stage");
 
 template <class GEO>
@@ -661,9 +691,13 @@ __device__ __forceinline__ void issuer_tiles_wm(const Cta& c, const GemmArgs& g,
 //         token over the tile's 128 output columns, e4m3 bytes and scales out, tile announced in f->ready.
 // MODE 2: blocks 0 / 1 = output columns [0,128) / [128,256) of the tile; bf16 out in the tile-blocked layout,
 //         then the per-(token, column tile) counters and the combine of the tokens this CTA completes.
-template <int MODE, class GEO>
-__device__ __forceinline__ void epilogue_tiles_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, TileRange tr,
-                                                  uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, bool& ok) {
+// One tile; false: a wait gave up (the code is in the status word).  SHARED: the tile runs inside the large-tile
+// kernel, between tiles of the other orientation -- its accumulators are the first 64 columns of the two
+// 256-column buffers of that kernel, handed over through the same two barriers, and its staging is the first
+// 512 bytes of the warp's own TMA staging area.
+template <int MODE, bool FUSED, class GEO, bool SHARED>
+__device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, int m_tile, int n,
+                                                 uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter) {
     GemmCtrl* ctrl = c.ctrl;
     const int warp = c.warp, lane = c.lane;
     const int th = (warp - 4) >> 2;          // which 16 of the tile's 32 token rows
@@ -671,234 +705,248 @@ __device__ __forceinline__ void epilogue_tiles_wm(const Cta& c, const GemmArgs& 
     // (lane l of quadrant q holds weight row 32 q + l of each 128-row block)
     const uint32_t t_lane = c.tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + th * 16;
     const size_t row_cap = static_cast<size_t>(g.row_cap);
-    uint32_t* amax_x = reinterpret_cast<uint32_t*>(c.amax_x);   // [2 parities][2 token halves][4 quadrants][16]
+    uint32_t* amax_x = reinterpret_cast<uint32_t*>(c.amax_x);   // [2 parities][256]: [2 token halves][4 quadrants][16] used
     const int num_kb = g.num_kb;
-    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
-        const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
-        const int e = __ldcg(g.tile_expert + m_tile);
-        const int rows_valid = __ldcg(g.tile_rows + m_tile);
-        const int sblocks = g.w_rows_per_expert / 128;
-        const float* ws0;  // weight-scale rows of block 0 / block 1
-        const float* ws1;
-        if (MODE == 1) {
-            ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.gate_row0 / 128 + n) * num_kb;
-            ws1 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.up_row0 / 128 + n) * num_kb;
-        } else {
-            ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + 2 * n) * num_kb;
-            ws1 = ws0 + num_kb;
-        }
-        float acc[32];  // [0,16): block 0, [16,32): block 1, for tokens 16 th .. 16 th + 15
+    const int e = __ldcg(g.tile_expert + m_tile);
+    const int rows_valid = __ldcg(g.tile_rows + m_tile);
+    const int sblocks = g.w_rows_per_expert / 128;
+    const float* ws0;  // weight-scale rows of block 0 / block 1
+    const float* ws1;
+    if (MODE == 1) {
+        ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.gate_row0 / 128 + n) * num_kb;
+        ws1 = g.w_scale + (static_cast<size_t>(e) * sblocks + g.up_row0 / 128 + n) * num_kb;
+    } else {
+        ws0 = g.w_scale + (static_cast<size_t>(e) * sblocks + 2 * n) * num_kb;
+        ws1 = ws0 + num_kb;
+    }
+    float acc[32];  // [0,16): block 0, [16,32): block 1, for tokens 16 th .. 16 th + 15
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc[j] = 0.0f;
+    for (int j = 0; j < 32; ++j) acc[j] = 0.0f;
 
-        float s0 = __ldg(ws0), s1 = __ldg(ws1);
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
-            const float w0 = s0, w1 = s1;
-            if (kb + 1 < num_kb) {
-                s0 = __ldg(ws0 + kb + 1);
-                s1 = __ldg(ws1 + kb + 1);
-            }
-            const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph, c.abort_flag, c.limit))) {
-                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                ok = false;
-                break;
-            }
-            tc_fence_after();
-            // the MMAs of this K-block have finished, hence its stage -- tokens, weights and scales -- had landed
-            const float4* sp = reinterpret_cast<const float4*>(c.scale_ring + (it % GEO::SCALE_SLOTS) * GEO::A_ROWS + th * 16);
-            float sa[16];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const float4 x = sp[q];
-                sa[4 * q] = x.x;
-                sa[4 * q + 1] = x.y;
-                sa[4 * q + 2] = x.z;
-                sa[4 * q + 3] = x.w;
-            }
-            float v[32];
-            tmem_ld16x2(t_lane + s * WM_BUF_COLS, t_lane + s * WM_BUF_COLS + WM_TOKENS, v);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[s]));
-#pragma unroll
-            for (int t = 0; t < 16; ++t) {
-                acc[t] = fmaf(v[t], sa[t] * w0, acc[t]);
-                acc[16 + t] = fmaf(v[16 + t], sa[t] * w1, acc[16 + t]);
-            }
+    float s0 = __ldg(ws0), s1 = __ldg(ws1);
+    for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        const float w0 = s0, w1 = s1;
+        if (kb + 1 < num_kb) {
+            s0 = __ldg(ws0 + kb + 1);
+            s1 = __ldg(ws1 + kb + 1);
         }
-        if (!ok) break;
+        const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph, c.abort_flag, c.limit))) {
+            if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+            return false;
+        }
+        tc_fence_after();
+        // the MMAs of this K-block have finished, hence its stage -- tokens, weights and scales -- had landed
+        const float4* sp = reinterpret_cast<const float4*>(c.scale_ring + (it % GEO::SCALE_SLOTS) * GEO::A_ROWS + th * 16);
+        float sa[16];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float4 x = sp[q];
+            sa[4 * q] = x.x;
+            sa[4 * q + 1] = x.y;
+            sa[4 * q + 2] = x.z;
+            sa[4 * q + 3] = x.w;
+        }
+        float v[32];
+        const uint32_t buf = SHARED ? (it & 1) : s, t_buf = t_lane + buf * (SHARED ? G_TILE_N : WM_BUF_COLS);
+        tmem_ld16x2(t_buf, t_buf + WM_TOKENS, v);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+            acc[t] = fmaf(v[t], sa[t] * w0, acc[t]);
+            acc[16 + t] = fmaf(v[16 + t], sa[t] * w1, acc[16 + t]);
+        }
+    }
 
-        const int tile_row0 = __ldcg(g.tile_row0 + m_tile);
-        const size_t row0 = static_cast<size_t>(tile_row0) + th * 16;  // padded row of this thread's token 0
-        const int valid = min(16, rows_valid - th * 16);                     // tokens of this thread that exist
-        if (MODE == 1) {
-            float cc[16];
-            uint32_t wmax[16];
+    const int tile_row0 = SHARED ? m_tile * TILE_M : __ldcg(g.tile_row0 + m_tile);
+    const size_t row0 = static_cast<size_t>(tile_row0) + th * 16;  // padded row of this thread's token 0
+    const uint32_t wst_off = (warp - 4) * (SHARED ? G_STORE_WARP_BYTES : 512);  // this warp's staging
+    if (SHARED) {  // the warp's last TMA store may still be reading the area
+        if (lane == 0) bulk_wait_read_all();
+        __syncwarp();
+    }
+    const int valid = min(16, rows_valid - th * 16);                     // tokens of this thread that exist
+    if (MODE == 1) {
+        float cc[16];
+        uint32_t wmax[16];
 #pragma unroll
-            for (int t = 0; t < 16; ++t) {
-                const float gt = acc[t];
-                cc[t] = __fdividef(gt, 1.0f + __expf(-gt)) * acc[16 + t];
-                // |x| as an integer orders like the float: the warp's maximum over its 32 output columns
-                wmax[t] = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(cc[t])));
-            }
-            const uint32_t par = tile_iter & 1;
-            uint32_t* xq = amax_x + ((par * 2 + th) * 4) * 16;
-            {
-                uint32_t mine = 0;
+        for (int t = 0; t < 16; ++t) {
+            const float gt = acc[t];
+            cc[t] = __fdividef(gt, 1.0f + __expf(-gt)) * acc[16 + t];
+            // |x| as an integer orders like the float: the warp's maximum over its 32 output columns
+            wmax[t] = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(cc[t])));
+        }
+        const uint32_t par = tile_iter & 1;
+        // (inside the half of the exchange area that belongs to this parity in the other orientation as well)
+        uint32_t* xq = amax_x + par * (2 * TILE_M) + th * 64;
+        {
+            uint32_t mine = 0;
 #pragma unroll
-                for (int t = 0; t < 16; ++t)
-                    if (lane == t) mine = wmax[t];
-                if (lane < 16) xq[quad * 16 + lane] = mine;
-            }
-            const uint32_t xbar = smem_u32(&ctrl->amax_bar[par]);
-            mbar_arrive(xbar);
-            if (!__all_sync(0xffffffffu, mbar_wait(xbar, (tile_iter >> 1) & 1, c.abort_flag, c.limit))) {
-                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                ok = false;
-                break;
-            }
-            ++tile_iter;
-            // lane t < 16 owns the scale of token t's 128-column block; everybody fetches its reciprocal
-            float my_sc = 1.0f, my_inv = 1.0f;
-            if (lane < 16) {
-                const volatile uint32_t* xv = xq + lane;
-                const float amax = __uint_as_float(max(max(xv[0], xv[16]), max(xv[32], xv[48])));
-                my_sc = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 448.0f);
-                my_inv = __frcp_rn(my_sc);
-            }
-            // Narrow global stores are slow (a warp's 32 single bytes cost tens of clocks): the codes are
-            // transposed through this warp's 512 bytes of staging, [16 tokens][32 columns], and leave as
-            // 16-byte stores -- lane l carries 16 columns of token l / 2.
-            uint8_t* wst = c.store_stage + (warp - 4) * 512;
+            for (int t = 0; t < 16; ++t)
+                if (lane == t) mine = wmax[t];
+            if (lane < 16) xq[quad * 16 + lane] = mine;
+        }
+        const uint32_t xbar = smem_u32(&ctrl->amax_bar[par]);
+        mbar_arrive(xbar);
+        if (!__all_sync(0xffffffffu, mbar_wait(xbar, (tile_iter >> 1) & 1, c.abort_flag, c.limit))) {
+            if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+            return false;
+        }
+        ++tile_iter;
+        // lane t < 16 owns the scale of token t's 128-column block; everybody fetches its reciprocal
+        float my_sc = 1.0f, my_inv = 1.0f;
+        if (lane < 16) {
+            const volatile uint32_t* xv = xq + lane;
+            const float amax = __uint_as_float(max(max(xv[0], xv[16]), max(xv[32], xv[48])));
+            my_sc = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 448.0f);
+            my_inv = __frcp_rn(my_sc);
+        }
+        // Narrow global stores are slow (a warp's 32 single bytes cost tens of clocks): the codes are
+        // transposed through this warp's 512 bytes of staging, [16 tokens][32 columns], and leave as
+        // 16-byte stores -- lane l carries 16 columns of token l / 2.
+        uint8_t* wst = c.store_stage + wst_off;
 #pragma unroll
-            for (int t = 0; t < 16; ++t) {
-                const float inv_sc = __shfl_sync(0xffffffffu, my_inv, t);
-                wst[t * 32 + lane] =
-                    static_cast<uint8_t>(__nv_cvt_float_to_fp8(cc[t] * inv_sc, __NV_SATFINITE, __NV_E4M3));
-            }
-            __syncwarp();
-            if ((lane >> 1) < valid)
-                *reinterpret_cast<uint4*>(g.out_fp8 + (row0 + (lane >> 1)) * g.out_cols + n * 128 + quad * 32 + (lane & 1) * 16) =
-                    *reinterpret_cast<const uint4*>(wst + (lane >> 1) * 32 + (lane & 1) * 16);
-            if (quad == 0 && lane < valid) g.out_scale_t[static_cast<size_t>(n) * row_cap + row0 + lane] = my_sc;
-            __syncwarp();
+        for (int t = 0; t < 16; ++t) {
+            const float inv_sc = __shfl_sync(0xffffffffu, my_inv, t);
+            wst[t * 32 + lane] =
+                static_cast<uint8_t>(__nv_cvt_float_to_fp8(cc[t] * inv_sc, __NV_SATFINITE, __NV_E4M3));
+        }
+        __syncwarp();
+        if ((lane >> 1) < valid)
+            *reinterpret_cast<uint4*>(g.out_fp8 + (row0 + (lane >> 1)) * g.out_cols + n * 128 + quad * 32 + (lane & 1) * 16) =
+                *reinterpret_cast<const uint4*>(wst + (lane >> 1) * 32 + (lane & 1) * 16);
+        if (quad == 0 && lane < valid) g.out_scale_t[static_cast<size_t>(n) * row_cap + row0 + lane] = my_sc;
+        __syncwarp();
+        // (The rows are read by copy engines, of other CTAs or of the next kernel: plain stores here,
+        // asynchronous-proxy loads there.)
+        fence_proxy_async();
+        if (FUSED) {
             // Announce the tile: every thread's stores are fenced before the epilogue warps meet, and the
-            // announcing thread fences once more behind the barrier.  (The rows are read by other CTAs' copy
-            // engines: plain stores here, asynchronous-proxy loads there.)
-            fence_proxy_async();
+            // announcing thread fences once more behind the barrier.
             __threadfence();
             if (!epilogue_rendezvous(c, sync_iter)) {
                 if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                ok = false;
-                break;
+                return false;
             }
             if (warp == 4 && lane == 0) {
                 __threadfence();
                 atomicAdd(f->ready + m_tile, 1);
             }
-        } else {
-            // bf16 out through this warp's 512 bytes of staging, eight tokens x 32 columns at a time, so that
-            // the rows leave as 16-byte stores: lane l carries 8 columns of token l / 4 (half of a 32-byte
-            // group of the tile-blocked layout)
-            __nv_bfloat16* wst = reinterpret_cast<__nv_bfloat16*>(c.store_stage + (warp - 4) * 512);
+        }
+    } else {
+        // bf16 out through this warp's 512 bytes of staging, eight tokens x 32 columns at a time, so that
+        // the rows leave as 16-byte stores: lane l carries 8 columns of token l / 4 (half of a 32-byte
+        // group of the tile-blocked layout)
+        __nv_bfloat16* wst = reinterpret_cast<__nv_bfloat16*>(c.store_stage + wst_off);
 #pragma unroll
-            for (int j = 0; j < 2; ++j) {
+        for (int j = 0; j < 2; ++j) {
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
+            for (int h = 0; h < 2; ++h) {
 #pragma unroll
-                    for (int t = 0; t < 8; ++t) wst[t * 32 + lane] = __float2bfloat16_rn(acc[j * 16 + h * 8 + t]);
-                    __syncwarp();
-                    const int t = h * 8 + (lane >> 2), ch0 = quad * 32 + (lane & 3) * 8;
-                    if (t < valid)
-                        *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(g.out_bf16) +
-                                                  y_block_offset(static_cast<int>(row0) + t, n * 16 + j * 8 + (ch0 >> 4), g.n_tiles) +
-                                                  (ch0 & 15) * 2) =
-                            *reinterpret_cast<const uint4*>(wst + (lane >> 2) * 32 + (lane & 3) * 8);
-                    __syncwarp();
-                }
-            }
-            // Stage 4 without a kernel of its own.  Once the tile is stored and fenced, the thread of each valid
-            // row bumps the counter of (its token, this column tile); whoever brings it to the token's number of
-            // local slots knows that all of the token's rows for these 256 columns are in memory and sums
-            // them, in routing order, exactly as combine_kernel does.
-            __threadfence();
-            if (!epilogue_rendezvous(c, sync_iter)) {
-                if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
-                ok = false;
-                break;
-            }
-            {
-                // epilogue warp w looks after the rows w, w + 8, w + 16, w + 24 of the tile (lanes 0..3), so up
-                // to eight completed tokens are summed at the same time
-                int tok = -1;
-                bool last = false;
-                const int r_mine = (warp - 4) + 8 * lane;
-                if (lane < 4 && r_mine < rows_valid) {
-                    tok = __ldcg(f->row_token + tile_row0 + r_mine);
-                    __threadfence();
-                    const int before = atomicAdd(f->tok_done + static_cast<size_t>(tok) * g.n_tiles + n, 1);
-                    last = before == __ldcg(f->tok_nlocal + tok) - 1;
-                }
-                uint32_t todo = __ballot_sync(0xffffffffu, last);
-                if (todo) __threadfence();
-                while (todo) {
-                    const int src = __ffs(todo) - 1;
-                    todo &= todo - 1;
-                    const int t = __shfl_sync(0xffffffffu, tok, src);
-                    // lane l owns columns n*256 + 8 l .. + 8: half of the 32-byte group n*16 + l/2.  All loads
-                    // first, then the sum in routing order.
-                    const int4 ra = __ldcg(reinterpret_cast<const int4*>(f->slot_to_row) + 2 * t);
-                    const int4 rb = __ldcg(reinterpret_cast<const int4*>(f->slot_to_row) + 2 * t + 1);
-                    const float4 wa = __ldcg(reinterpret_cast<const float4*>(f->topk_w) + 2 * t);
-                    const float4 wb = __ldcg(reinterpret_cast<const float4*>(f->topk_w) + 2 * t + 1);
-                    const int rr[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
-                    const float ww[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
-                    uint4 u[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        if (rr[j] >= 0)
-                            u[j] = __ldcg(reinterpret_cast<const uint4*>(
-                                reinterpret_cast<const uint8_t*>(g.out_bf16) +
-                                y_block_offset(rr[j], n * 16 + (lane >> 1), g.n_tiles) + (lane & 1) * 16));
-                    float o[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) o[i] = 0.0f;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        if (rr[j] < 0) continue;
-                        const uint32_t uu[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            o[2 * i] = fmaf(ww[j], __uint_as_float(uu[i] << 16), o[2 * i]);
-                            o[2 * i + 1] = fmaf(ww[j], __uint_as_float(uu[i] & 0xffff0000u), o[2 * i + 1]);
-                        }
-                    }
-                    uint32_t p[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const __nv_bfloat162 pr = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
-                        p[i] = *reinterpret_cast<const uint32_t*>(&pr);
-                    }
-                    *reinterpret_cast<uint4*>(f->out + static_cast<size_t>(t) * f->H + n * G_TILE_N + lane * 8) =
-                        make_uint4(p[0], p[1], p[2], p[3]);
-                }
+                for (int t = 0; t < 8; ++t) wst[t * 32 + lane] = __float2bfloat16_rn(acc[j * 16 + h * 8 + t]);
+                __syncwarp();
+                const int t = h * 8 + (lane >> 2), ch0 = quad * 32 + (lane & 3) * 8;
+                if (t < valid)
+                    *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(g.out_bf16) +
+                                              y_block_offset(static_cast<int>(row0) + t, n * 16 + j * 8 + (ch0 >> 4), g.n_tiles) +
+                                              (ch0 & 15) * 2) =
+                        *reinterpret_cast<const uint4*>(wst + (lane >> 2) * 32 + (lane & 3) * 8);
+                __syncwarp();
             }
         }
+        // Stage 4 without a kernel of its own.  Once the tile is stored and fenced, the thread of each valid
+        // row bumps the counter of (its token, this column tile); whoever brings it to the token's number of
+        // local slots knows that all of the token's rows for these 256 columns are in memory and sums
+        // them, in routing order, exactly as combine_kernel does.
+        if (!FUSED) return true;  // (one GEMM per launch: the combine is a kernel of its own)
+        __threadfence();
+        if (!epilogue_rendezvous(c, sync_iter)) {
+            if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+            return false;
+        }
+        {
+            // epilogue warp w looks after the rows w, w + 8, w + 16, w + 24 of the tile (lanes 0..3), so up
+            // to eight completed tokens are summed at the same time
+            int tok = -1;
+            bool last = false;
+            const int r_mine = (warp - 4) + 8 * lane;
+            if (lane < 4 && r_mine < rows_valid) {
+                tok = __ldcg(f->row_token + tile_row0 + r_mine);
+                __threadfence();
+                const int before = atomicAdd(f->tok_done + static_cast<size_t>(tok) * g.n_tiles + n, 1);
+                last = before == __ldcg(f->tok_nlocal + tok) - 1;
+            }
+            uint32_t todo = __ballot_sync(0xffffffffu, last);
+            if (todo) __threadfence();
+            while (todo) {
+                const int src = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const int t = __shfl_sync(0xffffffffu, tok, src);
+                // lane l owns columns n*256 + 8 l .. + 8: half of the 32-byte group n*16 + l/2.  All loads
+                // first, then the sum in routing order.
+                const int4 ra = __ldcg(reinterpret_cast<const int4*>(f->slot_to_row) + 2 * t);
+                const int4 rb = __ldcg(reinterpret_cast<const int4*>(f->slot_to_row) + 2 * t + 1);
+                const float4 wa = __ldcg(reinterpret_cast<const float4*>(f->topk_w) + 2 * t);
+                const float4 wb = __ldcg(reinterpret_cast<const float4*>(f->topk_w) + 2 * t + 1);
+                const int rr[8] = {ra.x, ra.y, ra.z, ra.w, rb.x, rb.y, rb.z, rb.w};
+                const float ww[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+                uint4 u[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (rr[j] >= 0)
+                        u[j] = __ldcg(reinterpret_cast<const uint4*>(
+                            reinterpret_cast<const uint8_t*>(g.out_bf16) +
+                            y_block_offset(rr[j], n * 16 + (lane >> 1), g.n_tiles) + (lane & 1) * 16));
+                float o[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) o[i] = 0.0f;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (rr[j] < 0) continue;
+                    const uint32_t uu[4] = {u[j].x, u[j].y, u[j].z, u[j].w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        o[2 * i] = fmaf(ww[j], __uint_as_float(uu[i] << 16), o[2 * i]);
+                        o[2 * i + 1] = fmaf(ww[j], __uint_as_float(uu[i] & 0xffff0000u), o[2 * i + 1]);
+                    }
+                }
+                uint32_t p[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const __nv_bfloat162 pr = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+                    p[i] = *reinterpret_cast<const uint32_t*>(&pr);
+                }
+                *reinterpret_cast<uint4*>(f->out + static_cast<size_t>(t) * f->H + n * G_TILE_N + lane * 8) =
+                    make_uint4(p[0], p[1], p[2], p[3]);
+            }
+        }
+    }
+    return true;
+}
+
+template <int MODE, bool FUSED, class GEO>
+__device__ __forceinline__ void epilogue_tiles_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, TileRange tr,
+                                                  uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, bool& ok) {
+    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+        const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
+        ok = epilogue_tile_wm<MODE, FUSED, GEO, false>(c, g, f, m_tile, n, it, tile_iter, sync_iter);
     }
 }
 
 // One GEMM per launch.
 template <int MODE>
 __global__ void __launch_bounds__(G_THREADS, 1)
-grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const __grid_constant__ CUtensorMap tmOut, const GemmArgs g) {
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAs,
+                    const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmOut, const GemmArgs g) {
     extern __shared__ uint8_t smem_raw[];
     using GEO = GeomFull;
     Cta c;
     gemm_cta_setup<GEO>(c, smem_raw, 1);
     if (c.warp == 0 && c.lane == 0) {
         tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmAs);
         tma_prefetch_desc(&tmB);
         if (MODE == 1) tma_prefetch_desc(&tmOut);
     }
@@ -919,7 +967,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (c.warp < 4) {
         reg_dealloc<40>();
         if (c.warp == 0 && c.lane == 0) {
-            producer_tiles<MODE, false, GEO>(c, &tmA, &tmB, g, nullptr, 0, tr, it, ok);
+            producer_tiles<MODE, false, GEO>(c, &tmA, &tmB, g, nullptr, 0, tr, it, ok, &tmAs);
             producer_drain<GEO>(c, g.status, it);
         } else if ((c.warp == 1 || c.warp == 2) && c.lane == 0) {
             issuer_tiles<GEO>(c, g, tr, c.warp - 1, it, ok);
@@ -1008,8 +1056,8 @@ fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_consta
     } else {
         reg_alloc<232>();
         uint32_t tile_iter = 0, sync_iter = 0;
-        epilogue_tiles_wm<1, GEO>(c, g1, &f, tr1, it, tile_iter, sync_iter, ok);
-        epilogue_tiles_wm<2, GEO>(c, g2, &f, tr2, it, tile_iter, sync_iter, ok);
+        epilogue_tiles_wm<1, true, GEO>(c, g1, &f, tr1, it, tile_iter, sync_iter, ok);
+        epilogue_tiles_wm<2, true, GEO>(c, g2, &f, tr2, it, tile_iter, sync_iter, ok);
     }
 
     tc_fence_before();

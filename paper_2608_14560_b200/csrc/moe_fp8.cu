@@ -107,7 +107,7 @@ struct moe_fp8_handle_s {
     uint8_t* ws;
     size_t ws_bytes;
     EncodeTiledFn encode;
-    CUtensorMap tm_a1, tm_a2, tm_a2_small, tm_a2_store, tm_w13, tm_w2;
+    CUtensorMap tm_a1, tm_a2, tm_a1_small, tm_a2_small, tm_a2_store, tm_w13, tm_w2;
     const void* w13_cached;
     const void* w2_cached;
     bool stage_timing;
@@ -116,6 +116,7 @@ struct moe_fp8_handle_s {
     long long fault_wait_limit;
     cudaEvent_t ev[NUM_STAGES_MAX + 1];
     int fused_max_tokens;   // batches of at most this many tokens take the fused kernel (0: never)
+    int short_tile_min_tokens;   // batches of at least this many tokens run short row tiles with the weights on M (0: never)
     unsigned long long fused_calls;
     // moe_fp8_forward_host_async: copy streams and the events that order the two staging sets
     bool pipe_ready;
@@ -285,6 +286,7 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     h->L = make_layout(*cfg);
     h->sm_count = sms;
     h->fused_max_tokens = F_DEFAULT_MAX_TOKENS;
+    h->short_tile_min_tokens = SHORT_TILE_MIN_TOKENS;
     h->fused_calls = 0;
     h->fault_skip_it = -1;
     h->fault_wait_limit = WAIT_LIMIT_CLOCKS;
@@ -329,6 +331,8 @@ int moe_fp8_set_workspace(moe_fp8_handle_t h, void* ws, size_t bytes) {
     if (!encode_2d(h, &h->tm_a1, h->ws + h->L.a1, h->L.row_cap, h->cfg.hidden, 1, 128, TILE_M,
                    CU_TENSOR_MAP_SWIZZLE_128B) ||
         !encode_2d(h, &h->tm_a2, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate, 1, 128, TILE_M,
+                   CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !encode_2d(h, &h->tm_a1_small, h->ws + h->L.a1, h->L.row_cap, h->cfg.hidden, 1, 128, GeomSmall::A_ROWS,
                    CU_TENSOR_MAP_SWIZZLE_128B) ||
         !encode_2d(h, &h->tm_a2_small, h->ws + h->L.a2, h->L.row_cap, h->cfg.intermediate, 1, 128, GeomSmall::A_ROWS,
                    CU_TENSOR_MAP_SWIZZLE_128B) ||
@@ -536,12 +540,13 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
             mark();
         }
         // stage 3a: GEMM1 + SwiGLU + re-quantisation
+        if (h->short_tile_min_tokens > 0 && T >= h->short_tile_min_tokens) g1.wm_rows = g2.wm_rows = WM_TOKENS;
         MOE_LAUNCH(grouped_gemm_kernel<1>, h->sm_count, G_THREADS, GeomFull::SMEM_BYTES, stream, pdl, h->tm_a1,
-                   h->tm_w13, h->tm_a2_store, g1);
+                   h->tm_a1_small, h->tm_w13, h->tm_a2_store, g1);
         mark();
         // stage 3b: GEMM2
         MOE_LAUNCH(grouped_gemm_kernel<2>, h->sm_count, G_THREADS, GeomFull::SMEM_BYTES, stream, pdl, h->tm_a2,
-                   h->tm_w2, h->tm_a2_store, g2);
+                   h->tm_a2_small, h->tm_w2, h->tm_a2_store, g2);
         mark();
         {  // stage 4: weighted combine back to token order
             const int grid = min(T, h->sm_count * 16);
@@ -564,6 +569,12 @@ int moe_fp8_debug_set_fault(moe_fp8_handle_t h, int skip_iteration, long long wa
     if (!h || wait_clocks < 0) return MOE_FP8_ERR_BAD_ARG;
     h->fault_skip_it = skip_iteration < 0 ? -1 : skip_iteration;
     h->fault_wait_limit = wait_clocks == 0 ? WAIT_LIMIT_CLOCKS : wait_clocks;
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_debug_set_short_tiles(moe_fp8_handle_t h, int min_tokens) {
+    if (!h || min_tokens < 0) return MOE_FP8_ERR_BAD_ARG;
+    h->short_tile_min_tokens = min_tokens;
     return MOE_FP8_OK;
 }
 
