@@ -344,6 +344,30 @@ def test_from_hidden_benchmark_shapes(cuda_device, cfg, n_sample):
     assert S > 0
 
 
+# ---- row tiles of at most 32 rows inside the large-tile GEMM kernels: weights on the M side of the MMAs ------
+@pytest.mark.parametrize("tokens,kw", [(100, {}), (200, {"skew": True}), (700, {}), (1111, {"skew": True}),
+                                       (3000, {"local_expert_offset": 160})])
+def test_short_row_tiles_are_bit_identical_to_full_row_tiles(cuda_device, tokens, kw):
+    # the same forward with every row tile worked on as a full 128-row tile (hook off) and with the short ones
+    # (an expert's last tile of at most 32 rows) taken the other way round, full and short tiles interleaved
+    # in every CTA's work list
+    wl = _wl(tokens, seed=500 + tokens, **kw)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device)
+    eng.debug_set_short_tiles(0)
+    want = eng.forward(inp).clone()
+    eng.debug_set_short_tiles(1)
+    got = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert eng.status() == 0
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    dbg = eng.debug_export(tokens, rows=False)
+    counts = dbg["expert_count"].cpu().numpy()
+    assert ((counts % 128 > 0) & (counts % 128 <= 32)).any(), "no short row tile in this workload"
+    run_and_compare(wl, cuda_device, inp=inp, eng=eng)
+    eng.close()
+
+
 # ---- batches of at most 80 tokens: gather, both GEMMs and the combine as one kernel; up to 16 tokens that ----
 # ---- kernel also routes and permutes (every CTA for itself), and the forward is a single launch -------------
 @pytest.mark.parametrize("tokens,kw", [(1, {}), (5, {}), (12, {}), (13, {}), (16, {"local_expert_offset": 64}),
