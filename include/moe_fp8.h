@@ -196,6 +196,15 @@ int moe_fp8_debug_export(moe_fp8_handle_t h, int T, int* topk_idx, float* topk_w
 int moe_fp8_set_small_batch_fusion(moe_fp8_handle_t h, int enable);
 
 /*
+ * Batches of at most 4 tokens with so few tiles that most SMs would idle: the fused kernel cuts every tile's K
+ * range into up to eight parts for different CTAs.  A part stores its per-K-block partial sums unscaled; the CTA
+ * that stores a tile's last part (found with a counter, nobody waits) applies the scales K-block after K-block
+ * in the order of the unsplit tile and finishes the tile, so results are bit-identical.  On by default; this
+ * hook turns it off (enable = 0) for the test that compares the two.
+ */
+int moe_fp8_debug_set_k_split(moe_fp8_handle_t h, int enable);
+
+/*
  * Inside the two large-tile GEMM kernels a row tile that holds at most 32 rows (an expert's short last tile) is
  * worked on with the operands swapped -- weights on the M side of the MMAs, the 32 token rows on N, a 64-column
  * accumulator -- instead of as a full 128-row tile: same arithmetic, bit-identical results, less tensor and

@@ -20,7 +20,7 @@ EXPORTS = (
     "moe_fp8_get_stage_times", "moe_fp8_expert_histogram_static", "moe_fp8_debug_set_fault",
     "moe_fp8_debug_sigmoid", "moe_fp8_forward_from_hidden", "moe_fp8_debug_export_inputs",
     "moe_fp8_set_small_batch_fusion", "moe_fp8_forward_host_async", "moe_fp8_host_sync",
-    "moe_fp8_debug_set_short_tiles",
+    "moe_fp8_debug_set_short_tiles", "moe_fp8_debug_set_k_split",
 )
 
 
@@ -87,6 +87,8 @@ def load_library() -> C.CDLL:
         lib.moe_fp8_expert_histogram_static.restype = C.c_int
         lib.moe_fp8_set_small_batch_fusion.argtypes = [vp, C.c_int]
         lib.moe_fp8_set_small_batch_fusion.restype = C.c_int
+        lib.moe_fp8_debug_set_k_split.argtypes = [vp, C.c_int]
+        lib.moe_fp8_debug_set_k_split.restype = C.c_int
         lib.moe_fp8_debug_set_short_tiles.argtypes = [vp, C.c_int]
         lib.moe_fp8_debug_set_short_tiles.restype = C.c_int
         lib.moe_fp8_debug_set_fault.argtypes = [vp, C.c_int, C.c_longlong]
@@ -235,6 +237,11 @@ class MoeFp8:
         kernel up to the default limit (80 tokens; a single launch per forward up to 16 tokens); 2..256 = the
         fused kernel up to that many tokens."""
         self._check(self.lib.moe_fp8_set_small_batch_fusion(self.handle, int(enable)))
+
+    def debug_set_k_split(self, enable: bool):
+        """moe_fp8_debug_set_k_split: batches of at most 4 tokens may cut a tile's K range over several CTAs
+        (default on)."""
+        self._check(self.lib.moe_fp8_debug_set_k_split(self.handle, int(enable)))
 
     def debug_set_short_tiles(self, min_tokens: int):
         """moe_fp8_debug_set_short_tiles: batch size from which row tiles of at most 32 rows run with the weights

@@ -159,7 +159,16 @@ struct FusedArgs {
     PermuteMeta meta;
     int* counters_next;           // the counter set of the NEXT fused call, zeroed by CTA 0 of this one
     int num_counters;
+    // K split of very small batches (T <= SPLIT_MAX_TOKENS, few tiles): the parts of a tile store their per-K-block
+    // partial sums here, [tile][K-block][weight-row block][128 rows][4 tokens] fp32 per GEMM, and count themselves
+    float* raw[2];
+    int* part_done[2];            // [tiles] per GEMM, zero at launch (part of the counter set)
+    int split;                    // 1: the split may be used by this call
 };
+constexpr int SPLIT_MAX_TOKENS = 4;                       // rows of a tile whose K range may be split
+constexpr int SPLIT_MAX_TILES = 74;                       // a split needs at least two CTAs per tile
+constexpr int SPLIT_RAW_FLOATS = 2 * SPLIT_MAX_TOKENS * 128;  // per tile and K-block
+constexpr int SPLIT_MAX_KB = 64;                          // K-blocks of a GEMM whose tiles may be split
 
 struct GemmCtrl {
     uint64_t full[G_MAX_STAGES];   // stage filled (TMA transaction bytes)
@@ -170,6 +179,7 @@ struct GemmCtrl {
     uint64_t sync_bar[2];      // fused kernel: rendezvous of the epilogue warps at the end of a tile
     uint32_t tmem_slot;
     int abort_flag;
+    int split_last;            // fused kernel, K split: this CTA stored the last part of the tile
 };
 static_assert(sizeof(GemmCtrl) <= G_CTRL_BYTES, "control block too large");
 
@@ -202,6 +212,20 @@ struct Cta {
 struct TileRange {
     int first, count, stride;
 };
+
+// Very small batches of the fused kernel: a tile's K range is cut into `parts` pieces of `len` K-blocks that
+// different CTAs work on (see epilogue_tile_wm).  parts = 1: a work item is a whole tile.
+struct KSplit {
+    int parts, len;
+};
+__device__ __forceinline__ KSplit ksplit_none(int num_kb) { return KSplit{1, num_kb}; }
+// as many parts as keep every CTA at one item at most, eight at most
+__device__ __forceinline__ KSplit ksplit_for(int num_kb, int tiles, int grid, bool allowed) {
+    int want = (allowed && tiles > 0) ? grid / tiles : 1;
+    want = want < 1 ? 1 : (want > 8 ? 8 : want);
+    const int len = (num_kb + want - 1) / want;
+    return KSplit{(num_kb + len - 1) / len, len};
+}
 
 template <class GEO>
 __device__ __forceinline__ void gemm_cta_setup(Cta& c, uint8_t* smem_raw, int full_count) {
@@ -244,9 +268,12 @@ __device__ __forceinline__ void gemm_cta_setup(Cta& c, uint8_t* smem_raw, int fu
 template <int MODE, bool FUSED, class GEO>
 __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* tmA, const CUtensorMap* tmB,
                                                const GemmArgs& g, const FusedArgs* f, int ready_target, TileRange tr,
-                                               uint32_t& it, bool& ok, const CUtensorMap* tmA_short = nullptr) {
+                                               uint32_t& it, bool& ok, const CUtensorMap* tmA_short = nullptr,
+                                               KSplit ks = KSplit{1, 1 << 30}) {
     GemmCtrl* ctrl = c.ctrl;
-    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+    for (int item = tr.first; item < tr.count && ok; item += tr.stride) {
+        const int tile = item / ks.parts, kb0 = (item - tile * ks.parts) * ks.len;
+        const int kb1 = min(g.num_kb, kb0 + ks.len);
         const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
         const int wrow = __ldcg(g.tile_expert + m_tile) * g.w_rows_per_expert;
         const int row0 = FUSED ? __ldcg(g.tile_row0 + m_tile) : m_tile * TILE_M;
@@ -293,14 +320,14 @@ __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* 
                          a_sc + static_cast<size_t>(kb) * g.row_cap, wm ? WM_TOKENS * 4 : GEO::SCALE_BYTES, bar);
             tma_load_2d(c.smem_base + s * GEO::STAGE_BYTES, wm ? tmA_short : tmA, kb * G_BLOCK_K, row0, bar);
         };
-        int kb = 0;
+        int kb = kb0;
         if (FUSED && MODE == 2) {
             // The tile's A rows are GEMM1's output and must have been stored; its weights need not wait for
             // that, so the B tiles of the first K-blocks go out before the counter is looked at.
-            const int npre = g.num_kb < GEO::STAGES ? g.num_kb : GEO::STAGES;
+            const int npre = kb1 - kb0 < GEO::STAGES ? kb1 - kb0 : GEO::STAGES;
             for (int k = 0; k < npre && ok; ++k) {
                 ok = claim(it + k);
-                if (ok) load_b(it + k, k);
+                if (ok) load_b(it + k, kb0 + k);
             }
             if (!ok) break;
             if (!wait_counter(f->ready + m_tile, ready_target, c.abort_flag, c.limit)) {
@@ -309,11 +336,11 @@ __device__ __forceinline__ void producer_tiles(const Cta& c, const CUtensorMap* 
                 break;
             }
             fence_proxy_async();  // the rows were stored by other CTAs' copy engines; order our copies behind the acquire
-            for (int k = 0; k < npre; ++k) load_a(it + k, k);
+            for (int k = 0; k < npre; ++k) load_a(it + k, kb0 + k);
             it += npre;
-            kb = npre;
+            kb = kb0 + npre;
         }
-        for (; kb < g.num_kb && ok; ++kb, ++it) {
+        for (; kb < kb1 && ok; ++kb, ++it) {
             ok = claim(it);
             if (!ok) break;
             if (!(FUSED && MODE == 1)) load_a(it, kb);
@@ -402,12 +429,14 @@ __device__ __forceinline__ void issuer_drain(const Cta& c, uint32_t mine, bool o
 // past the tile's valid rows are zero-filled; the stage holds only these 32 rows (see Geometry).  Each lane's arrival on full[s] is triggered by the completion of its copies.
 template <class GEO>
 __device__ __forceinline__ void gather_tiles(const Cta& c, const GemmArgs& g, const FusedArgs& f, TileRange tr,
-                                             uint32_t& it, bool& ok) {
+                                             uint32_t& it, bool& ok, KSplit ks) {
     GemmCtrl* ctrl = c.ctrl;
     const int lane = c.lane, sub = lane >> 3, chunk = lane & 7;
     const uint32_t dst_even = sub * 128 + ((chunk ^ sub) << 4);
     const uint32_t dst_odd = sub * 128 + ((chunk ^ (sub + 4)) << 4);
-    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+    for (int item = tr.first; item < tr.count && ok; item += tr.stride) {
+        const int tile = item / ks.parts, kb0 = (item - tile * ks.parts) * ks.len;
+        const int kb1 = min(g.num_kb, kb0 + ks.len);
         const int m_tile = tile / g.n_tiles;
         const int rows_valid = __ldcg(g.tile_rows + m_tile);
         // token of row `lane` (scale copy) and source rows of this lane's eight chunks
@@ -424,7 +453,7 @@ __device__ __forceinline__ void gather_tiles(const Cta& c, const GemmArgs& g, co
             sc_src = f.scale_layout ? f.hidden_scale + my_tok : f.hidden_scale + static_cast<size_t>(my_tok) * g.num_kb;
             sc_step = f.scale_layout ? static_cast<size_t>(f.T) : 1;
         }
-        for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
             const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
             if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, c.abort_flag, c.limit))) {
                 if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_PRODUCER);
@@ -447,10 +476,12 @@ __device__ __forceinline__ void gather_tiles(const Cta& c, const GemmArgs& g, co
 }
 // GEMM2 tiles: the producer fetches everything; the lanes only keep the arrival count of full[s] uniform.
 template <class GEO>
-__device__ __forceinline__ void gather_idle_tiles(const Cta& c, const GemmArgs& g, TileRange tr, uint32_t& it, bool& ok) {
+__device__ __forceinline__ void gather_idle_tiles(const Cta& c, const GemmArgs& g, TileRange tr, uint32_t& it, bool& ok,
+                                                  KSplit ks) {
     GemmCtrl* ctrl = c.ctrl;
-    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
-        for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+    for (int item = tr.first; item < tr.count && ok; item += tr.stride) {
+        const int kb0 = (item % ks.parts) * ks.len, kb1 = min(g.num_kb, kb0 + ks.len);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
             const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
             if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctrl->done[s]), ph ^ 1, c.abort_flag, c.limit))) {
                 ok = false;
@@ -474,7 +505,8 @@ __device__ __forceinline__ bool epilogue_rendezvous(const Cta& c, uint32_t& n) {
 
 template <int MODE, bool FUSED, class GEO, bool SHARED>
 __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, int m_tile, int n,
-                                                 uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter);
+                                                 uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, int kb0 = 0,
+                                                 int kb1 = -1, int parts = 1);
 
 // ---------------- epilogue warps ----------------
 // MODE 1: gate/up projection + SwiGLU + re-quantisation; tmOut describes the e4m3 output [row_cap, I] for
@@ -651,13 +683,14 @@ static_assert(G_MAX_STAGES * WM_BUF_COLS <= static_cast<int>(G_TMEM_COLS), "one 
 
 template <class GEO>
 __device__ __forceinline__ void issuer_tiles_wm(const Cta& c, const GemmArgs& g, TileRange tr, uint32_t mine,
-                                                uint32_t& it, bool& ok) {
+                                                uint32_t& it, bool& ok, KSplit ks) {
     static_assert(GEO::A_ROWS == WM_TOKENS, "the token slot of a stage is the MMA's N operand");
     static_assert(GEO::SCALE_SLOTS >= 2 * GEO::STAGES + 1, "the gather may be two pipelines ahead of the epilogue");
     GemmCtrl* ctrl = c.ctrl;
     const uint32_t idesc = umma_idesc_f8(TILE_M, WM_TOKENS);
-    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
-        for (int kb = 0; kb < g.num_kb; ++kb, ++it) {
+    for (int item = tr.first; item < tr.count && ok; item += tr.stride) {
+        const int kb0 = (item % ks.parts) * ks.len, kb1 = min(g.num_kb, kb0 + ks.len);
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
             if ((it & 1) != mine) continue;
             const uint32_t s = it % GEO::STAGES, ph = (it / GEO::STAGES) & 1;
             const uint32_t tok_addr = c.smem_base + s * GEO::STAGE_BYTES;
@@ -695,9 +728,15 @@ __device__ __forceinline__ void issuer_tiles_wm(const Cta& c, const GemmArgs& g,
 // kernel, between tiles of the other orientation -- its accumulators are the first 64 columns of the two
 // 256-column buffers of that kernel, handed over through the same two barriers, and its staging is the first
 // 512 bytes of the warp's own TMA staging area.
+// parts > 1 (fused kernel, batches of at most SPLIT_MAX_TOKENS tokens with few tiles): this call covers the
+// K-blocks [kb0, kb1) only.  It stores every K-block's partial sums as they come out of the tensor memory, not
+// yet multiplied by the scales; the CTA that stores the last part of a tile -- found with a counter, nobody
+// waits -- then runs the whole promotion from the stored partial sums, K-block after K-block in the one order
+// the unsplit tile uses, and finishes the tile.  Every fp32 operation is the one of the unsplit tile.
 template <int MODE, bool FUSED, class GEO, bool SHARED>
 __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, int m_tile, int n,
-                                                 uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter) {
+                                                 uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, int kb0, int kb1,
+                                                 int parts) {
     GemmCtrl* ctrl = c.ctrl;
     const int warp = c.warp, lane = c.lane;
     const int th = (warp - 4) >> 2;          // which 16 of the tile's 32 token rows
@@ -723,10 +762,17 @@ __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g
 #pragma unroll
     for (int j = 0; j < 32; ++j) acc[j] = 0.0f;
 
-    float s0 = __ldg(ws0), s1 = __ldg(ws1);
-    for (int kb = 0; kb < num_kb; ++kb, ++it) {
+    const bool split = FUSED && parts > 1;
+    const int kb_end = kb1 < 0 ? num_kb : kb1;
+    const int tile_row0 = SHARED ? m_tile * TILE_M : __ldcg(g.tile_row0 + m_tile);
+    float4* raw = nullptr;  // this tile's stored partial sums (four tokens each): this thread's weight row
+    if (FUSED && split)
+        raw = reinterpret_cast<float4*>(f->raw[MODE - 1] + static_cast<size_t>(m_tile * g.n_tiles + n) * num_kb * SPLIT_RAW_FLOATS) +
+              quad * 32 + lane;
+    float s0 = __ldg(ws0 + kb0), s1 = __ldg(ws1 + kb0);
+    for (int kb = kb0; kb < kb_end; ++kb, ++it) {
         const float w0 = s0, w1 = s1;
-        if (kb + 1 < num_kb) {
+        if (kb + 1 < kb_end) {
             s0 = __ldg(ws0 + kb + 1);
             s1 = __ldg(ws1 + kb + 1);
         }
@@ -753,6 +799,13 @@ __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
+        if (FUSED && split) {
+            if (th == 0) {  // (all four token columns; those past the tile's rows are never used)
+                raw[(kb * 2 + 0) * 128] = make_float4(v[0], v[1], v[2], v[3]);
+                raw[(kb * 2 + 1) * 128] = make_float4(v[16], v[17], v[18], v[19]);
+            }
+            continue;
+        }
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
             acc[t] = fmaf(v[t], sa[t] * w0, acc[t]);
@@ -760,7 +813,80 @@ __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g
         }
     }
 
-    const int tile_row0 = SHARED ? m_tile * TILE_M : __ldcg(g.tile_row0 + m_tile);
+    if (FUSED && split) {
+        // count this part; the last one goes on, the others are done with the tile
+        __threadfence();
+        if (!epilogue_rendezvous(c, sync_iter)) {
+            if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+            return false;
+        }
+        if (warp == 4 && lane == 0) {
+            __threadfence();
+            const int before = atomicAdd(f->part_done[MODE - 1] + m_tile * g.n_tiles + n, 1);
+            *reinterpret_cast<volatile int*>(&ctrl->split_last) = (before == parts - 1);
+        }
+        if (!epilogue_rendezvous(c, sync_iter)) {
+            if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+            return false;
+        }
+        if (!*reinterpret_cast<volatile int*>(&ctrl->split_last)) return true;
+        __threadfence();
+        // The finisher.  The scales of the tile's (at most four) tokens and of the two weight-row blocks go to
+        // shared memory first (the row-maximum exchange area is free here: every warp has left the previous
+        // tile); then the warps of token half 0 promote block 0 and those of half 1 block 1, K-block after
+        // K-block, and half 1 hands its sums to half 0 through the staging area.
+        float* sa_s = c.amax_x;                                   // [num_kb][4]
+        float* w_s = c.amax_x + SPLIT_MAX_TOKENS * num_kb;        // [2][num_kb]
+        static_assert(G_AMAX_BYTES >= (SPLIT_MAX_TOKENS + 2) * SPLIT_MAX_KB * 4, "scales of a tile's K-blocks");
+        for (int i = threadIdx.x - 128; i < SPLIT_MAX_TOKENS * num_kb; i += G_EPI_WARPS * 32) {
+            const int kb = i / SPLIT_MAX_TOKENS, t = i - kb * SPLIT_MAX_TOKENS;
+            float v = 0.0f;
+            if (t < rows_valid) {
+                if (MODE == 1) {
+                    const int tok = __ldcg(f->row_token + tile_row0 + t);
+                    v = __ldcg(f->scale_layout ? f->hidden_scale + static_cast<size_t>(kb) * f->T + tok
+                                               : f->hidden_scale + static_cast<size_t>(tok) * num_kb + kb);
+                } else {
+                    v = __ldcg(g.a_scale_t + static_cast<size_t>(kb) * row_cap + tile_row0 + t);
+                }
+            }
+            sa_s[i] = v;
+        }
+        for (int i = threadIdx.x - 128; i < 2 * num_kb; i += G_EPI_WARPS * 32)
+            w_s[i] = __ldg((i < num_kb ? ws0 : ws1 - num_kb) + i);
+        if (!epilogue_rendezvous(c, sync_iter)) {
+            if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+            return false;
+        }
+        float4 a4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        {
+            const float4* rp = raw + th * 128;
+            const float* wp = w_s + th * num_kb;
+#pragma unroll 28
+            for (int kb = 0; kb < num_kb; ++kb) {
+                const float4 r = __ldcg(rp + kb * 2 * 128);
+                const float4 sa = *reinterpret_cast<const float4*>(sa_s + kb * SPLIT_MAX_TOKENS);
+                const float w = wp[kb];
+                a4.x = fmaf(r.x, sa.x * w, a4.x);
+                a4.y = fmaf(r.y, sa.y * w, a4.y);
+                a4.z = fmaf(r.z, sa.z * w, a4.z);
+                a4.w = fmaf(r.w, sa.w * w, a4.w);
+            }
+        }
+        float4* xchg = reinterpret_cast<float4*>(c.store_stage);  // [128 weight rows]: half 0's warps read their own staging
+        if (th == 1) xchg[quad * 32 + lane] = a4;
+        if (!epilogue_rendezvous(c, sync_iter)) {
+            if (lane == 0) raise(ctrl, g.status, DEV_TIMEOUT_EPILOGUE);
+            return false;
+        }
+        if (th == 0) {
+            const float4 b4 = xchg[quad * 32 + lane];
+            acc[0] = a4.x, acc[1] = a4.y, acc[2] = a4.z, acc[3] = a4.w;
+            acc[16] = b4.x, acc[17] = b4.y, acc[18] = b4.z, acc[19] = b4.w;
+        }
+        __syncwarp();
+    }
+
     const size_t row0 = static_cast<size_t>(tile_row0) + th * 16;  // padded row of this thread's token 0
     const uint32_t wst_off = (warp - 4) * (SHARED ? G_STORE_WARP_BYTES : 512);  // this warp's staging
     if (SHARED) {  // the warp's last TMA store may still be reading the area
@@ -928,10 +1054,13 @@ __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g
 
 template <int MODE, bool FUSED, class GEO>
 __device__ __forceinline__ void epilogue_tiles_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, TileRange tr,
-                                                  uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, bool& ok) {
-    for (int tile = tr.first; tile < tr.count && ok; tile += tr.stride) {
+                                                  uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, bool& ok,
+                                                  KSplit ks) {
+    for (int item = tr.first; item < tr.count && ok; item += tr.stride) {
+        const int tile = item / ks.parts, kb0 = (item - tile * ks.parts) * ks.len;
         const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
-        ok = epilogue_tile_wm<MODE, FUSED, GEO, false>(c, g, f, m_tile, n, it, tile_iter, sync_iter);
+        ok = epilogue_tile_wm<MODE, FUSED, GEO, false>(c, g, f, m_tile, n, it, tile_iter, sync_iter, kb0,
+                                                       min(g.num_kb, kb0 + ks.len), ks.parts);
     }
 }
 
@@ -1031,8 +1160,14 @@ fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_consta
 
     // The CTA's work list: its GEMM1 tiles, then its GEMM2 tiles; the grid-strided numbering runs on from one
     // phase into the next, so the CTAs that had no GEMM1 tile take the first GEMM2 tiles.
+    // Very small batches with few tiles: a tile's K range is cut into parts for different CTAs (KSplit).
     const int grid = static_cast<int>(gridDim.x), m_tiles = __ldcg(g1.num_m_tiles);
-    const int n1 = m_tiles * g1.n_tiles, n2 = m_tiles * g2.n_tiles;
+    const bool may_split = f.split && f.T <= SPLIT_MAX_TOKENS && g1.num_kb <= SPLIT_MAX_KB && g2.num_kb <= SPLIT_MAX_KB;
+    const KSplit ks1 = ksplit_for(g1.num_kb, m_tiles * g1.n_tiles, grid, may_split && m_tiles * g1.n_tiles <= SPLIT_MAX_TILES);
+    // (GEMM2's K range is too short for it: counting the parts and the finisher's pass over the stored partial sums
+    // cost 5-6 us per tile, which 16 K-blocks do not win back; measured 1-2 us slower)
+    const KSplit ks2 = ksplit_none(g2.num_kb);
+    const int n1 = m_tiles * g1.n_tiles * ks1.parts, n2 = m_tiles * g2.n_tiles * ks2.parts;
     const TileRange tr1 = {static_cast<int>(blockIdx.x), n1, grid};
     const TileRange tr2 = {((static_cast<int>(blockIdx.x) - n1) % grid + grid) % grid, n2, grid};
     uint32_t it = 0;
@@ -1041,23 +1176,23 @@ fused_small_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_consta
     if (c.warp < 4) {
         reg_dealloc<40>();
         if (c.warp == 0 && c.lane == 0) {
-            producer_tiles<1, true, GEO>(c, &tmA2, &tmB1, g1, &f, 0, tr1, it, ok);
-            producer_tiles<2, true, GEO>(c, &tmA2, &tmB2, g2, &f, g1.n_tiles, tr2, it, ok);
+            producer_tiles<1, true, GEO>(c, &tmA2, &tmB1, g1, &f, 0, tr1, it, ok, nullptr, ks1);
+            producer_tiles<2, true, GEO>(c, &tmA2, &tmB2, g2, &f, g1.n_tiles, tr2, it, ok, nullptr, ks2);
             producer_drain<GEO>(c, g1.status, it);
         } else if ((c.warp == 1 || c.warp == 2) && c.lane == 0) {
-            issuer_tiles_wm<GEO>(c, g1, tr1, c.warp - 1, it, ok);
-            issuer_tiles_wm<GEO>(c, g2, tr2, c.warp - 1, it, ok);
+            issuer_tiles_wm<GEO>(c, g1, tr1, c.warp - 1, it, ok, ks1);
+            issuer_tiles_wm<GEO>(c, g2, tr2, c.warp - 1, it, ok, ks2);
             issuer_drain(c, c.warp - 1, ok);
         } else if (c.warp == 3) {
-            gather_tiles<GEO>(c, g1, f, tr1, it, ok);
-            gather_idle_tiles<GEO>(c, g2, tr2, it, ok);
+            gather_tiles<GEO>(c, g1, f, tr1, it, ok, ks1);
+            gather_idle_tiles<GEO>(c, g2, tr2, it, ok, ks2);
             cp_async_wait_all();  // nothing may still be landing in shared memory when the CTA exits
         }
     } else {
         reg_alloc<232>();
         uint32_t tile_iter = 0, sync_iter = 0;
-        epilogue_tiles_wm<1, true, GEO>(c, g1, &f, tr1, it, tile_iter, sync_iter, ok);
-        epilogue_tiles_wm<2, true, GEO>(c, g2, &f, tr2, it, tile_iter, sync_iter, ok);
+        epilogue_tiles_wm<1, true, GEO>(c, g1, &f, tr1, it, tile_iter, sync_iter, ok, ks1);
+        epilogue_tiles_wm<2, true, GEO>(c, g2, &f, tr2, it, tile_iter, sync_iter, ok, ks2);
     }
 
     tc_fence_before();

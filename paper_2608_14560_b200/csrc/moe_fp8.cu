@@ -30,7 +30,7 @@ inline size_t align_up(size_t x, size_t a = WS_ALIGN) { return (x + a - 1) / a *
 
 struct WsLayout {
     size_t topk_idx, topk_w, block_hist, expert_count, expert_offset, padded_offset, tile_expert, tile_rows,
-        num_m_tiles, slot_to_row, row_to_slot, row_token, tok_nlocal, st_expert, st_row0, st_rows, num_st, counters, num_counters, max_st, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
+        num_m_tiles, slot_to_row, row_to_slot, row_token, tok_nlocal, st_expert, st_row0, st_rows, num_st, counters, num_counters, max_st, raw1, raw2, status, a1, a1_scale_t, a2, a2_scale_t, y, stage_hidden,
         stage_scale, stage_logits, stage_out, stage2_hidden, stage2_scale, stage2_logits, stage2_out, total;
     int row_cap, max_m_tiles, max_blocks;
 };
@@ -72,8 +72,12 @@ WsLayout make_layout(const moe_fp8_config& c) {
     L.st_rows = take(L.max_st * 4);
     L.num_st = take(4);
     // (a batch the fused kernel takes has at most EL + F_MAX_TOKENS * 8 / 32 sub-tiles)
-    L.num_counters = std::min<size_t>(L.max_st, EL + F_MAX_TOKENS / 4) + static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N);
+    // (then the parts stored per tile by the K split of very small batches, per GEMM)
+    L.num_counters = std::min<size_t>(L.max_st, EL + F_MAX_TOKENS / 4) + static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N) +
+                     2 * SPLIT_MAX_TILES;
     L.counters = take(2 * L.num_counters * 4);
+    L.raw1 = take(static_cast<size_t>(SPLIT_MAX_TILES) * (H / 128) * SPLIT_RAW_FLOATS * 4);
+    L.raw2 = take(static_cast<size_t>(SPLIT_MAX_TILES) * (I / 128) * SPLIT_RAW_FLOATS * 4);
     L.status = take(8);  // device status word, then the ticket counter of route_permute_kernel
     L.a1 = take(rc * H);
     L.a1_scale_t = take(rc * (H / 128) * 4);
@@ -116,6 +120,7 @@ struct moe_fp8_handle_s {
     long long fault_wait_limit;
     cudaEvent_t ev[NUM_STAGES_MAX + 1];
     int fused_max_tokens;   // batches of at most this many tokens take the fused kernel (0: never)
+    bool k_split;           // fused kernel: very small batches may cut a tile's K range over several CTAs
     int short_tile_min_tokens;   // batches of at least this many tokens run short row tiles with the weights on M (0: never)
     unsigned long long fused_calls;
     // moe_fp8_forward_host_async: copy streams and the events that order the two staging sets
@@ -286,6 +291,7 @@ int moe_fp8_create(const moe_fp8_config* cfg, moe_fp8_handle_t* out) {
     h->L = make_layout(*cfg);
     h->sm_count = sms;
     h->fused_max_tokens = F_DEFAULT_MAX_TOKENS;
+    h->k_split = true;
     h->short_tile_min_tokens = SHORT_TILE_MIN_TOKENS;
     h->fused_calls = 0;
     h->fault_skip_it = -1;
@@ -504,7 +510,12 @@ int moe_fp8_forward(moe_fp8_handle_t h, int T, const void* hidden_fp8, const flo
         f.topk_w = topk_w;
         f.tok_nlocal = m.tok_nlocal;
         f.ready = counters;
-        f.tok_done = counters + (h->L.num_counters - static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N));
+        f.tok_done = counters + (h->L.num_counters - 2 * SPLIT_MAX_TILES - static_cast<size_t>(F_MAX_TOKENS) * (H / G_TILE_N));
+        f.part_done[0] = counters + (h->L.num_counters - 2 * SPLIT_MAX_TILES);
+        f.part_done[1] = f.part_done[0] + SPLIT_MAX_TILES;
+        f.raw[0] = at<float>(h, h->L.raw1);
+        f.raw[1] = at<float>(h, h->L.raw2);
+        f.split = h->k_split ? 1 : 0;
         // the fused kernel works on sub-tiles of at most 32 rows
         g1.num_m_tiles = g2.num_m_tiles = m.num_st;
         g1.tile_expert = g2.tile_expert = m.st_expert;
@@ -569,6 +580,12 @@ int moe_fp8_debug_set_fault(moe_fp8_handle_t h, int skip_iteration, long long wa
     if (!h || wait_clocks < 0) return MOE_FP8_ERR_BAD_ARG;
     h->fault_skip_it = skip_iteration < 0 ? -1 : skip_iteration;
     h->fault_wait_limit = wait_clocks == 0 ? WAIT_LIMIT_CLOCKS : wait_clocks;
+    return MOE_FP8_OK;
+}
+
+int moe_fp8_debug_set_k_split(moe_fp8_handle_t h, int enable) {
+    if (!h) return MOE_FP8_ERR_BAD_ARG;
+    h->k_split = enable != 0;
     return MOE_FP8_OK;
 }
 

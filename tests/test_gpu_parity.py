@@ -344,6 +344,28 @@ def test_from_hidden_benchmark_shapes(cuda_device, cfg, n_sample):
     assert S > 0
 
 
+# ---- batches of at most 4 tokens: GEMM1's K range of every tile cut over several CTAs ------------------------
+@pytest.mark.parametrize("tokens,eloc,off,seed", [(1, 32, 0, 3), (2, 32, 0, 1), (3, 32, 0, 2), (4, 32, 0, 0), (4, 1, 7, 5),
+                                                  (4, 3, 5, 6), (4, 256, 0, 7), (1, 256, 0, 8)])
+def test_k_split_of_very_small_batches_is_bit_identical(cuda_device, tokens, eloc, off, seed):
+    # few tiles (the split is used) and, with all 256 experts local, many tiles (it is not); the full-size layer
+    # has 56 K-blocks per GEMM1 tile, i.e. parts of 7 to 28 K-blocks
+    dims = dataclasses.replace(syn.CONFIGS[0].dims, num_local_experts=eloc) if eloc <= 32 else dataclasses.replace(SMALL, num_local_experts=eloc)
+    wl = syn.Workload(f"k{tokens}", tokens, dims, 700 + seed, local_expert_offset=off)
+    inp = syn.make_inputs(wl, cuda_device)
+    eng = make_engine(wl, cuda_device)
+    eng.debug_set_k_split(False)
+    want = eng.forward(inp).clone()
+    eng.debug_set_k_split(True)
+    for _ in range(3):  # the part counters of one forward must not disturb the next
+        got = eng.forward(inp).clone()
+    torch.cuda.synchronize()
+    assert eng.status() == 0 and eng.last_launch_count() == 1
+    assert torch.equal(got.view(torch.int16), want.view(torch.int16))
+    run_and_compare(wl, cuda_device, inp=inp, eng=eng)
+    eng.close()
+
+
 # ---- row tiles of at most 32 rows inside the large-tile GEMM kernels: weights on the M side of the MMAs ------
 @pytest.mark.parametrize("tokens,kw", [(100, {}), (200, {"skew": True}), (700, {}), (1111, {"skew": True}),
                                        (3000, {"local_expert_offset": 160})])
@@ -429,9 +451,9 @@ def test_fused_kernel_with_a_raised_limit_cuts_experts_into_sub_tiles(cuda_devic
     eng.close()
 
 
-@pytest.mark.parametrize("tokens,launches", [(16, 1), (48, 2)])
-def test_a_wait_that_runs_out_in_the_fused_small_batch_kernel(cuda_device, tokens, launches):
-    wl = _wl(tokens, seed=43)
+@pytest.mark.parametrize("tokens,launches,eloc", [(16, 1, 32), (48, 2, 32), (3, 1, 256)])  # 3 tokens: K split
+def test_a_wait_that_runs_out_in_the_fused_small_batch_kernel(cuda_device, tokens, launches, eloc):
+    wl = _wl(tokens, dataclasses.replace(SMALL, num_local_experts=eloc), seed=43)
     inp = syn.make_inputs(wl, cuda_device)
     eng = make_engine(wl, cuda_device)
     want = eng.forward(inp).clone()
