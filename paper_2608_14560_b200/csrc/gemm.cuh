@@ -503,7 +503,7 @@ __device__ __forceinline__ bool epilogue_rendezvous(const Cta& c, uint32_t& n) {
     return ok;
 }
 
-template <int MODE, bool FUSED, class GEO, bool SHARED>
+template <int MODE, bool FUSED, class GEO, bool SHARED, bool SPLIT = false>
 __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, int m_tile, int n,
                                                  uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, int kb0 = 0,
                                                  int kb1 = -1, int parts = 1);
@@ -728,15 +728,16 @@ __device__ __forceinline__ void issuer_tiles_wm(const Cta& c, const GemmArgs& g,
 // kernel, between tiles of the other orientation -- its accumulators are the first 64 columns of the two
 // 256-column buffers of that kernel, handed over through the same two barriers, and its staging is the first
 // 512 bytes of the warp's own TMA staging area.
-// parts > 1 (fused kernel, batches of at most SPLIT_MAX_TOKENS tokens with few tiles): this call covers the
+// SPLIT (fused kernel, batches of at most SPLIT_MAX_TOKENS tokens with few tiles, parts > 1): this call covers the
 // K-blocks [kb0, kb1) only.  It stores every K-block's partial sums as they come out of the tensor memory, not
 // yet multiplied by the scales; the CTA that stores the last part of a tile -- found with a counter, nobody
 // waits -- then runs the whole promotion from the stored partial sums, K-block after K-block in the one order
 // the unsplit tile uses, and finishes the tile.  Every fp32 operation is the one of the unsplit tile.
-template <int MODE, bool FUSED, class GEO, bool SHARED>
+template <int MODE, bool FUSED, class GEO, bool SHARED, bool SPLIT>
 __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g, const FusedArgs* f, int m_tile, int n,
                                                  uint32_t& it, uint32_t& tile_iter, uint32_t& sync_iter, int kb0, int kb1,
                                                  int parts) {
+    static_assert(!SPLIT || FUSED, "only the fused kernel cuts K ranges");
     GemmCtrl* ctrl = c.ctrl;
     const int warp = c.warp, lane = c.lane;
     const int th = (warp - 4) >> 2;          // which 16 of the tile's 32 token rows
@@ -762,11 +763,10 @@ __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g
 #pragma unroll
     for (int j = 0; j < 32; ++j) acc[j] = 0.0f;
 
-    const bool split = FUSED && parts > 1;
     const int kb_end = kb1 < 0 ? num_kb : kb1;
     const int tile_row0 = SHARED ? m_tile * TILE_M : __ldcg(g.tile_row0 + m_tile);
     float4* raw = nullptr;  // this tile's stored partial sums (four tokens each): this thread's weight row
-    if (FUSED && split)
+    if (SPLIT)
         raw = reinterpret_cast<float4*>(f->raw[MODE - 1] + static_cast<size_t>(m_tile * g.n_tiles + n) * num_kb * SPLIT_RAW_FLOATS) +
               quad * 32 + lane;
     float s0 = __ldg(ws0 + kb0), s1 = __ldg(ws1 + kb0);
@@ -799,21 +799,21 @@ __device__ __forceinline__ bool epilogue_tile_wm(const Cta& c, const GemmArgs& g
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->tmem_empty[buf]));
-        if (FUSED && split) {
+        if (SPLIT) {
             if (th == 0) {  // (all four token columns; those past the tile's rows are never used)
                 raw[(kb * 2 + 0) * 128] = make_float4(v[0], v[1], v[2], v[3]);
                 raw[(kb * 2 + 1) * 128] = make_float4(v[16], v[17], v[18], v[19]);
             }
-            continue;
-        }
+        } else {
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
-            acc[t] = fmaf(v[t], sa[t] * w0, acc[t]);
-            acc[16 + t] = fmaf(v[16 + t], sa[t] * w1, acc[16 + t]);
+            for (int t = 0; t < 16; ++t) {
+                acc[t] = fmaf(v[t], sa[t] * w0, acc[t]);
+                acc[16 + t] = fmaf(v[16 + t], sa[t] * w1, acc[16 + t]);
+            }
         }
     }
 
-    if (FUSED && split) {
+    if (SPLIT) {
         // count this part; the last one goes on, the others are done with the tile
         __threadfence();
         if (!epilogue_rendezvous(c, sync_iter)) {
@@ -1059,8 +1059,11 @@ __device__ __forceinline__ void epilogue_tiles_wm(const Cta& c, const GemmArgs& 
     for (int item = tr.first; item < tr.count && ok; item += tr.stride) {
         const int tile = item / ks.parts, kb0 = (item - tile * ks.parts) * ks.len;
         const int m_tile = tile / g.n_tiles, n = tile - m_tile * g.n_tiles;
-        ok = epilogue_tile_wm<MODE, FUSED, GEO, false>(c, g, f, m_tile, n, it, tile_iter, sync_iter, kb0,
-                                                       min(g.num_kb, kb0 + ks.len), ks.parts);
+        // (two instantiations, so that the unsplit tile's loop carries nothing of the split)
+        ok = (FUSED && MODE == 1 && ks.parts > 1)
+                 ? epilogue_tile_wm<MODE, FUSED, GEO, false, FUSED && MODE == 1>(c, g, f, m_tile, n, it, tile_iter, sync_iter, kb0,
+                                                                                min(g.num_kb, kb0 + ks.len), ks.parts)
+                 : epilogue_tile_wm<MODE, FUSED, GEO, false, false>(c, g, f, m_tile, n, it, tile_iter, sync_iter);
     }
 }
 
